@@ -1,0 +1,490 @@
+#!/usr/bin/env python
+"""Benchmark of the LineAR hot path on B200: image tokens/s of compressed-KV decode attention.
+
+One "step" = one whole image generation of the batch through the hot path: reset, prefill append,
+then for every visual token and every layer one fused append+decode-attention launch, and at every
+line end the score/evict/compact launch of every layer.  Inputs are synthetic (seeded generator of
+paper_2512_04857_b200.workloads) and resident in HBM before the timed region; the per-line launch
+sequences are captured once into CUDA graphs and replayed.  All layers are cycled every token, so
+the working set (GBs) is far larger than L2.
+
+Prints ONE JSON line (see README for the keys).  `--impl reference` times the CPU oracle
+on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "image tokens/s of compressed-KV decode attention"
+UNIT = "image_tokens/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        if self.p is not None:
+            self.p.terminate()
+            try:
+                self.p.wait(timeout=5)
+            except Exception:
+                self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                 parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        load = [x for x in sm if x >= 0.5 * max(sm)] or sm
+        return {"sm_mhz": statistics.median(load), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------------
+def cpu_baseline(w, budget_s: float = 12.0, seed_units: int = 8):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload's independent units."""
+    import numpy as np
+    from oracle import lar_oracle as O
+    from paper_2512_04857_b200 import workloads as W
+    cores = os.cpu_count() or 1
+    cfg = O.cfg_from_workload(w)
+
+    def sample(n_units, first):
+        us = []
+        for i in range(n_units):
+            j = first + i
+            layer = j % w.n_layers
+            s = (j // w.n_layers) % w.batch
+            h = (j // (w.n_layers * w.batch)) % w.n_kv_heads
+            us.append(W.gen_unit(w, layer, s, h))
+        st = lambda key: np.stack([u[key].numpy() for u in us])
+        return st("q"), st("k"), st("v"), st("kc"), st("vc")
+
+    ins = sample(seed_units, 0)
+    t0 = time.perf_counter()
+    _, _, thr = O.run_units(cfg, *ins, want_out=False, want_kept=False)
+    t_probe = time.perf_counter() - t0
+    per_unit = t_probe / seed_units
+    n_units = int(min(max(seed_units, budget_s / max(per_unit, 1e-6)), 64 * cores, w.n_layers * w.n_units))
+    n_units = max(cores, (n_units // cores) * cores)
+    ins = sample(n_units, seed_units)
+    t0 = time.perf_counter()
+    _, _, thr = O.run_units(cfg, *ins, want_out=True, want_kept=True)
+    dt = time.perf_counter() - t0
+    units_per_image = w.n_layers * w.n_units / w.images
+    value = (n_units / units_per_image) * w.n_visual / dt
+    return {"value": value, "unit": UNIT, "cores": int(thr), "kind": "oracle",
+            "sample": f"{n_units} of {w.n_layers * w.n_units} independent (layer, sequence, kv-head) units of "
+                      f"'{w.name}', whole generation ({w.n_visual} tokens, line-end evictions), {dt:.1f} s",
+            "seconds": dt, "units": n_units}
+
+
+def run_reference(args):
+    from paper_2512_04857_b200 import workloads as W
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = W.WORKLOADS[args.workload]
+    vals = []
+    cb = None
+    for i in range(args.warmup + args.steps):
+        cb = cpu_baseline(w, budget_s=max(2.0, min(20.0, 90.0 / max(1, args.warmup + args.steps))))
+        if i >= args.warmup:
+            vals.append(cb)
+    value = sum(c["units"] for c in vals) / sum(c["seconds"] for c in vals) * vals[0]["value"] * vals[0]["seconds"] / vals[0]["units"]
+    ms = 1e3 * sum(c["seconds"] for c in vals) / len(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "sampled_units_per_step": vals[0]["units"]},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cb["cores"], "kind": "oracle",
+                             "sample": cb["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+class Runner:
+    """Device-resident inputs + per-line CUDA graphs of one workload."""
+
+    def __init__(self, w, dev, args, flags_extra=0):
+        import torch
+        from paper_2512_04857_b200 import lar, workloads as W
+        self.torch, self.lar, self.w, self.dev = torch, lar, w, dev
+        flags = lar.LAR_FLAG_NO_HOST_CHECKS | flags_extra
+        if not args.no_pdl:
+            flags |= lar.LAR_FLAG_PDL
+        self.cfg = lar.config_from_workload(w, flags=flags, kv_splits=args.kv_splits, warps_per_cta=args.warps,
+                                            stages=args.stages, page_tokens=args.page_tokens)
+        self.cache = lar.Cache(self.cfg, device=str(dev))
+        L, S, Hq, Hkv, d, n, h = w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.line_width, w.n_lines
+        dt = w.torch_dtype
+        self.q = torch.empty((h, n, L, S, Hq, d), dtype=dt, device=dev)
+        self.k = torch.empty((h, n, L, S, Hkv, d), dtype=dt, device=dev)
+        self.v = torch.empty((h, n, L, S, Hkv, d), dtype=dt, device=dev)
+        self.kc = torch.empty((L, S, Hkv, max(w.cond_len, 1), d), dtype=dt, device=dev)
+        self.vc = torch.empty_like(self.kc)
+        self.out = torch.empty((n, L, S, Hq, d), dtype=dt, device=dev)
+        for layer in range(L):
+            if w.cond_len:
+                a, b = W.gen_prefix(w, layer, dev)
+                self.kc[layer], self.vc[layer] = a, b
+            for line in range(h):
+                q, k, v = W.gen_tokens(w, layer, line * n, (line + 1) * n, dev)
+                self.q[line, :, layer], self.k[line, :, layer], self.v[line, :, layer] = q, k, v
+        torch.cuda.synchronize(dev)
+        self.graphs = None
+        self.launches_per_generation = 0
+
+    def _enqueue_line(self, line, with_line_end=True):
+        w, c = self.w, self.cache
+        if line == 0:
+            c.reset()
+            if w.cond_len:
+                for layer in range(w.n_layers):
+                    c.append_kv(layer, self.kc[layer], self.vc[layer], w.cond_len)
+        return self._enqueue_decode(line), (self._enqueue_line_end(line) if with_line_end else 0)
+
+    def _enqueue_decode(self, line):
+        w, c = self.w, self.cache
+        for t in range(w.line_width):
+            for layer in range(w.n_layers):
+                c.decode_step(layer, self.q[line, t, layer], self.k[line, t, layer], self.v[line, t, layer],
+                              self.out[t, layer])
+        return w.line_width * w.n_layers
+
+    def _enqueue_line_end(self, line):
+        w, c = self.w, self.cache
+        if line == w.n_lines - 1:
+            return 0
+        for layer in range(w.n_layers):
+            c.line_end_score_evict(layer)
+        return w.n_layers
+
+    def capture(self):
+        """Two graphs per line: A = (reset + prefill on line 0) + n x L fused decode steps, B = L line ends."""
+        torch = self.torch
+        self.graphs = []
+        s = torch.cuda.Stream(device=self.dev)
+        n0 = self.cache.launch_count()
+        with torch.cuda.stream(s):
+            for line in range(self.w.n_lines):
+                ga = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(ga, stream=s):
+                    if line == 0:
+                        self.cache.reset()
+                        if self.w.cond_len:
+                            for layer in range(self.w.n_layers):
+                                self.cache.append_kv(layer, self.kc[layer], self.vc[layer], self.w.cond_len)
+                    self._enqueue_decode(line)
+                gb = None
+                if line < self.w.n_lines - 1:
+                    gb = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(gb, stream=s):
+                        self._enqueue_line_end(line)
+                self.graphs.append((ga, gb))
+        torch.cuda.synchronize(self.dev)
+        self.launches_per_generation = self.cache.launch_count() - n0
+
+    def generation(self, events=None):
+        """Replay one whole image generation on the current stream; optionally record (start, end) events
+        around the decode part of every line."""
+        torch = self.torch
+        for line, (ga, gb) in enumerate(self.graphs):
+            if events is not None:
+                e0, e1 = events[line]
+                e0.record()
+                ga.replay()
+                e1.record()
+            else:
+                ga.replay()
+            if gb is not None:
+                gb.replay()
+
+    def eager_generation(self):
+        for line in range(self.w.n_lines):
+            self._enqueue_line(line)
+
+    def close(self):
+        self.graphs = None
+        self.cache.close()
+        self.q = self.k = self.v = self.out = None
+
+
+def time_generations(r: Runner, steps: int, warmup: int, dist=None, sampler=None):
+    torch = r.torch
+    dev = r.dev
+    for _ in range(warmup):
+        r.generation()
+    torch.cuda.synchronize(dev)
+    evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+            for _ in range(r.w.n_lines)] for _ in range(steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize(dev)
+    if sampler:
+        sampler.start()
+    start.record()
+    for s in range(steps):
+        r.generation(evs[s])
+    stop.record()
+    torch.cuda.synchronize(dev)
+    clocks = sampler.stop() if sampler else None
+    if dist is not None:
+        dist.barrier()
+    total_ms = start.elapsed_time(stop)
+    decode_ms = sum(e0.elapsed_time(e1) for step in evs for (e0, e1) in step)
+    n = r.w.line_width
+    half = r.w.n_lines // 2
+    first_ms = sum(e0.elapsed_time(e1) for step in evs for (e0, e1) in step[:half]) / (steps * half * n)
+    last_ms = sum(e0.elapsed_time(e1) for step in evs for (e0, e1) in step[half:]) / (steps * (r.w.n_lines - half) * n)
+    return total_ms, decode_ms, clocks, (first_ms, last_ms)
+
+
+def measure_e2e(w, dev, args, steps=1):
+    """Same metric through the host-buffer entry point: every layer-step copies q, k, v from pinned host
+    memory, runs the fused kernel and copies the output back (all inside the timed region)."""
+    import torch
+    from paper_2512_04857_b200 import lar, workloads as W
+    flags = lar.LAR_FLAG_NO_HOST_CHECKS
+    cfg = lar.config_from_workload(w, flags=flags, kv_splits=args.kv_splits, warps_per_cta=args.warps,
+                                   stages=args.stages, page_tokens=args.page_tokens)
+    cache = lar.Cache(cfg, device=str(dev))
+    L, S, Hq, Hkv, d, n, h = w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.line_width, w.n_lines
+    dt = w.torch_dtype
+    # one line of pinned host inputs, reused for every line (throughput does not depend on the values)
+    hq = torch.empty((n, L, S, Hq, d), dtype=dt).pin_memory()
+    hk = torch.empty((n, L, S, Hkv, d), dtype=dt).pin_memory()
+    hv = torch.empty((n, L, S, Hkv, d), dtype=dt).pin_memory()
+    ho = torch.empty((n, L, S, Hq, d), dtype=dt).pin_memory()
+    for layer in range(L):
+        q, k, v = W.gen_tokens(w, layer, 0, n, dev)
+        hq[:, layer], hk[:, layer], hv[:, layer] = q.cpu(), k.cpu(), v.cpu()
+    kc = torch.zeros((L, S, Hkv, max(w.cond_len, 1), d), dtype=dt, device=dev)
+    s = torch.cuda.Stream(device=dev)
+    graphs = []
+    with torch.cuda.stream(s):
+        for kind in ("line+end", "line"):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                for t in range(n):
+                    for layer in range(L):
+                        cache.decode_step_host(layer, hq[t, layer], hk[t, layer], hv[t, layer], ho[t, layer])
+                if kind == "line+end":
+                    for layer in range(L):
+                        cache.line_end_score_evict(layer)
+            graphs.append(g)
+
+        def gen():
+            cache.reset()
+            if w.cond_len:
+                for layer in range(L):
+                    cache.append_kv(layer, kc[layer], kc[layer], w.cond_len)
+            for line in range(h):
+                graphs[0 if line < h - 1 else 1].replay()
+        gen()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            gen()
+        e1.record()
+        torch.cuda.synchronize(dev)
+    ms = e0.elapsed_time(e1) / steps
+    bits = cache.poll_device_status()
+    cache.close()
+    qb = S * Hq * d * w.elt_bytes
+    kb = S * Hkv * d * w.elt_bytes
+    return {"ms": ms, "h2d": w.n_visual * L * (qb + 2 * kb), "d2h": w.n_visual * L * qb, "status_bits": bits}
+
+
+def run_ours(args):
+    import torch
+    from paper_2512_04857_b200 import lar, workloads as W
+    lar.lib()  # fail loudly if the CUDA library is missing
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group(backend="nccl", device_id=torch.device(f"cuda:{local}"))
+        dist = dist_mod
+    dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(dev)
+    peak, peak_kind = load_peaks()
+    w = W.WORKLOADS[args.workload]
+
+    def bench_workload(wl, steps, warmup, sample_clocks):
+        r = Runner(wl, dev, args)
+        r.capture()
+        sampler = ClockSampler(local) if sample_clocks else None
+        total_ms, decode_ms, clocks, halves = time_generations(r, steps, warmup, dist, sampler)
+        bits = r.cache.poll_device_status()
+        plan = r.cache.plan
+        res = {"ms_per_step": total_ms / steps, "decode_ms_per_step": decode_ms / steps, "clocks": clocks,
+               "launches": r.launches_per_generation, "status_bits": bits,
+               "plan": {"kv_splits": plan.kv_splits, "warps_per_cta": plan.warps_per_cta, "stages": plan.stages,
+                        "page_tokens": plan.page_tokens, "decode_smem_bytes": plan.decode_smem_bytes},
+               "per_token_ms_first_half": halves[0], "per_token_ms_last_half": halves[1]}
+        r.close()
+        torch.cuda.empty_cache()
+        return res
+
+    main = bench_workload(w, args.steps, args.warmup, True)
+    ms = torch.tensor([main["ms_per_step"], main["decode_ms_per_step"]], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    ms_step, ms_decode = float(ms[0]), float(ms[1])
+    value = world * w.images * w.n_visual / (ms_step * 1e-3)
+    kv_bytes = w.kv_bytes_per_generation()
+    n_decode = w.n_visual * w.n_layers
+    achieved = kv_bytes / (ms_decode * 1e-3) / 1e9
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "layers": w.n_layers, "sequences": w.batch, "images": w.images,
+                       "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+                       "storage": w.dtype, "prefix": w.cond_len, "grid": f"{w.n_lines}x{w.line_width}",
+                       "budget_lines": w.budget_lines, "anchor": w.anchor_len, "recent_lines": w.recent_lines,
+                       "launch": "cuda-graph per line, fused append+decode, PDL" if not args.no_pdl
+                       else "cuda-graph per line, fused append+decode",
+                       "l2": "inputs larger than L2: all layers cycled every token "
+                             f"({kv_bytes / n_decode / 1e6:.0f} MB per launch x {w.n_layers} layers)",
+                       "plan": main["plan"], "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
+            "clocks": main["clocks"],
+            "gpu_launches": main["launches"] * args.steps,
+            "roofline": {"bound": "hbm", "kernel": "decode_kernel (fused append + decode attention)",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_kind": f"of {peak_kind} copy bandwidth",
+                         "frac_of_8TBs": achieved / 8000.0,
+                         "algorithmic_bytes_per_launch": kv_bytes / n_decode,
+                         "avg_launch_us": ms_decode * 1e3 / n_decode, "traffic": None},
+            "sequence_tokens_per_s": world * w.batch * w.n_visual / (ms_step * 1e-3),
+            "line_end_ms_per_step": ms_step - ms_decode,
+            "per_token_ms": {"first_half": main["per_token_ms_first_half"], "last_half": main["per_token_ms_last_half"]},
+            "device_status_bits": main["status_bits"]}
+
+    if rank == 0 or dist is None:
+        pass
+    # ---- speedup over the library's own full-cache path on the same inputs
+    if not args.no_full:
+        full = bench_workload(w.full_cache(), max(1, min(args.steps, 2)), 1, False)
+        fm = torch.tensor([full["ms_per_step"]], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(fm, op=dist.ReduceOp.MAX)
+        line["full_cache"] = {"ms_per_step": float(fm[0]), "value": world * w.images * w.n_visual / (float(fm[0]) * 1e-3),
+                              "per_token_ms": {"first_half": full["per_token_ms_first_half"],
+                                               "last_half": full["per_token_ms_last_half"]}}
+        line["speedup_vs_full_cache"] = float(fm[0]) / ms_step
+    # ---- end to end through host buffers
+    if not args.no_e2e:
+        e = measure_e2e(w, dev, args)
+        em = torch.tensor([e["ms"]], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(em, op=dist.ReduceOp.MAX)
+        line["e2e"] = {"value": world * w.images * w.n_visual / (float(em[0]) * 1e-3), "unit": UNIT,
+                       "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"], "ms_per_step": float(em[0]),
+                       "api": "lar_decode_step_host (pinned host q,k,v -> device, kernel, out -> host) per layer-step"}
+    # ---- other benchmark shapes (not the headline line)
+    if args.also:
+        line["also"] = {}
+        for name in args.also.split(","):
+            w2 = W.WORKLOADS[name]
+            r2 = bench_workload(w2, max(1, min(args.steps, 3)), 1, False)
+            ach = w2.kv_bytes_per_generation() / (r2["decode_ms_per_step"] * 1e-3) / 1e9
+            line["also"][name] = {"value": world * w2.images * w2.n_visual / (r2["ms_per_step"] * 1e-3), "unit": UNIT,
+                                  "ms_per_step": r2["ms_per_step"], "roofline_achieved_gbs": ach,
+                                  "roofline_frac": ach / peak, "frac_of_8TBs": ach / 8000.0, "plan": r2["plan"]}
+    # ---- CPU oracle on the host cores (rank 0, N = 1 only)
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = {k: v for k, v in cpu_baseline(w).items() if k not in ("seconds", "units")}
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="janus_pro_7b")
+    ap.add_argument("--also", default="", help="comma-separated extra workloads reported under 'also'")
+    ap.add_argument("--kv-splits", type=int, default=0)
+    ap.add_argument("--warps", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--page-tokens", type=int, default=0)
+    ap.add_argument("--no-pdl", action="store_true")
+    ap.add_argument("--no-full", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,181 @@
+/*
+ * lar.h — C ABI of the LineAR hot path on one B200 (sm_100a).
+ *
+ * The library manages, per transformer layer, a per-head KV cache that is bounded to a few raster
+ * lines (paper Sec. 3.3) and computes the per-token decode attention over it (Sec. 3.1, Eq. 2).
+ * Every (layer, sequence, KV head) is an independent unit: its live cache is
+ *     [ C conditional tokens | N_init anchor tokens | retained mid tokens | r most recent lines ]
+ * and never holds more than C + B entries, B = budget_lines * line_width.
+ *
+ * General conventions
+ *   - All entry points return a lar_status_t; nothing throws or aborts.
+ *   - "device" pointers are CUDA device addresses on the device that was current at
+ *     lar_cache_create; "host" pointers are ordinary (preferably pinned) host addresses.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Hot-path
+ *     calls only enqueue work on it: no host synchronisation, no allocation.
+ *   - The caller owns every buffer it passes, including the slab; the library owns only host-side
+ *     bookkeeping.  Buffers must stay valid until the enqueued work has run.
+ *   - Sequences decode in lock-step (one visual token per call for the whole batch), as in the
+ *     paper's batched runs; lengths are nevertheless stored per unit in device memory.
+ *   - Tensor layouts are dense, row-major, innermost dimension head_dim:
+ *       q, out : [batch, n_q_heads, head_dim]            k, v : [batch, n_kv_heads, n_tokens, head_dim]
+ *     Query head hq uses KV head hq / (n_q_heads / n_kv_heads).
+ *   - Element type is bf16 or fp32 (config); logits, softmax and accumulation are fp32.
+ */
+#ifndef LAR_H_
+#define LAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lar_cache lar_cache_t; /* opaque host object; device state lives in the caller's slab */
+
+typedef enum {
+    LAR_OK = 0,
+    LAR_ERR_INVALID_ARG = 1,  /* null pointer, bad size, unsupported shape */
+    LAR_ERR_BAD_STATE = 2,    /* call order violates the decode protocol (see each call) */
+    LAR_ERR_CAPACITY = 3,     /* append beyond the n-token line buffer / beyond N tokens */
+    LAR_ERR_CUDA = 4,         /* a CUDA runtime call failed; lar_last_cuda_error() has its code */
+    LAR_ERR_NOMEM = 5,        /* slab too small / host allocation failed */
+    LAR_ERR_DEVICE_CHECK = 6  /* a kernel recorded a failed bounds / wait-limit check */
+} lar_status_t;
+
+typedef enum { LAR_BF16 = 0, LAR_FP32 = 1 } lar_dtype_t;
+
+/* config.flags */
+#define LAR_FLAG_NO_HOST_CHECKS 0x1u /* skip the host-side call-order checks (needed when calls are
+                                        captured once into a CUDA graph and replayed: the host-side
+                                        counters then no longer follow the device). Device-side
+                                        checks stay active. */
+#define LAR_FLAG_PDL 0x2u            /* launch decode kernels with programmatic dependent launch and
+                                        let them prefetch cached K/V before the preceding kernel on the
+                                        stream has finished.  Contract: the kernel enqueued on `stream`
+                                        immediately before a decode call of layer l does not write layer
+                                        l's cache (the library checks this for its own launches), and any
+                                        caller kernel using PDL waits on its own dependency before it
+                                        triggers its dependents. */
+#define LAR_FLAG_SHUFFLE_PAGES 0x4u  /* test hook: assign physical pages in a pseudo-random order */
+
+typedef struct lar_config {
+    uint32_t struct_size;  /* = sizeof(lar_config_t) */
+    int32_t n_layers;      /* L */
+    int32_t batch;         /* S: sequences, after classifier-free-guidance doubling */
+    int32_t n_q_heads;     /* Hq */
+    int32_t n_kv_heads;    /* Hkv, divides Hq; Hq/Hkv in {1,2,4,8} */
+    int32_t head_dim;      /* d: 64 or 128 */
+    int32_t dtype;         /* lar_dtype_t */
+    int32_t cond_len;      /* C: conditional prefix (Sec. 3.1 prefill); always kept, not counted in B */
+    int32_t line_width;    /* n: tokens per raster line, including a line-end token if the model has one */
+    int32_t n_lines;       /* h: N = h * n visual tokens per image (Sec. 3.3, 2D view) */
+    int32_t anchor_len;    /* N_init: the first N_init visual tokens are never evicted (Sec. 3.3) */
+    int32_t recent_lines;  /* r >= 1: the last r lines are never evicted (Sec. 3.3) */
+    int32_t budget_lines;  /* B / n (Sec. 3.3 "Cache Budget"); >= n_lines selects the full-cache path */
+    float softmax_scale;   /* 0 selects 1/sqrt(head_dim) (Eq. 2) */
+    int32_t page_tokens;   /* tokens per physical page: 16, 32 or 64; 0 selects 16 */
+    uint32_t flags;        /* LAR_FLAG_* */
+    int32_t kv_splits;     /* CTAs (one thread-block cluster) per unit in decode: 0 auto, else 1,2,4,8 */
+    int32_t warps_per_cta; /* decode warps per CTA: 0 auto, else 1..8 */
+    int32_t stages;        /* 16-row K/V stages in flight per warp: 0 auto, else 1..4 */
+    uint32_t page_seed;    /* seed of LAR_FLAG_SHUFFLE_PAGES */
+} lar_config_t;
+
+/* What lar_cache_create derived from a config (introspection; also usable without a GPU). */
+typedef struct lar_plan {
+    int32_t capacity;       /* slots per unit: C + min(B, N) */
+    int32_t pages_per_unit;
+    int32_t page_tokens;
+    int32_t mid_len;        /* M = B - N_init - r n at a compressing line end; 0 on the full-cache path */
+    int32_t kv_splits, warps_per_cta, stages;
+    int32_t decode_smem_bytes;
+    int32_t line_end_smem_bytes;
+    int32_t compressing;    /* 1 if budget_lines < n_lines */
+    uint64_t slab_bytes;
+} lar_plan_t;
+
+/* Validate a config and report the derived plan.  No CUDA call is made.
+ * Rejects (LAR_ERR_INVALID_ARG): Hq % Hkv != 0, group not in {1,2,4,8}, d not in {64,128}, r < 1,
+ * negative sizes, and compressing budgets with fewer than n mid candidates
+ * (B < N_init + (r+1) n) — the paper does not define the method there. */
+lar_status_t lar_plan_query(const lar_config_t* cfg, lar_plan_t* plan_out);
+
+/* Bytes of device memory the caller must provide for a cache of this config (0 if invalid).
+ * The slab holds the paged K/V pools of all layers, page tables, per-unit lengths, the slot ->
+ * original-position index maps, the guide queues (Eq. 8) and the last score vectors (Eq. 9). */
+size_t lar_cache_slab_bytes(const lar_config_t* cfg);
+
+/* Create a cache over a caller-allocated device slab (256-byte aligned, >= lar_cache_slab_bytes).
+ * Writes page tables and zeroes the state on the legacy default stream and synchronises once.
+ * *out is owned by the caller until lar_cache_destroy. */
+lar_status_t lar_cache_create(const lar_config_t* cfg, void* dev_slab, size_t slab_bytes, lar_cache_t** out);
+
+/* Forget all cached tokens of every layer (start of a new image).  Asynchronous on `stream`. */
+lar_status_t lar_cache_reset(lar_cache_t* c, void* stream);
+
+/* Cache append (Eq. 4).  k, v: device, [batch, n_kv_heads, n_tokens, head_dim].
+ * The first call on a layer after create/reset is the prefill (Sec. 3.1): n_tokens must equal C
+ * (skip it if C = 0).  Every later call appends one visual token (n_tokens = 1) and must be
+ * followed by lar_decode_attn of that layer before the next append.
+ * LAR_ERR_CAPACITY: the line's n-token buffer is full (a line-end call is due) or N tokens exist. */
+lar_status_t lar_append_kv(lar_cache_t* c, int layer, const void* k, const void* v, int n_tokens, void* stream);
+
+/* Decode attention (Eq. 2-3) of the token appended last: out = softmax(q K^T scale) V over every live
+ * entry of the unit (prefix + retained visual tokens + the new token), per query head.
+ * q, out: device, [batch, n_q_heads, head_dim].  Also stores q in the layer's guide queue (Eq. 8).
+ * LAR_ERR_BAD_STATE unless a visual token was appended to this layer since its last decode. */
+lar_status_t lar_decode_attn(lar_cache_t* c, int layer, const void* q, void* out, void* stream);
+
+/* lar_append_kv(n_tokens = 1) + lar_decode_attn fused into one kernel launch (Eq. 4 then Eq. 2).
+ * k, v: device, [batch, n_kv_heads, head_dim]. */
+lar_status_t lar_decode_step(lar_cache_t* c, int layer, const void* q, const void* k, const void* v,
+                             void* out, void* stream);
+
+/* lar_decode_step with HOST buffers: copies q, k, v to a staging area of the slab, runs the fused
+ * kernel and copies `out` back, all asynchronously on `stream` (use pinned memory). */
+lar_status_t lar_decode_step_host(lar_cache_t* c, int layer, const void* q_host, const void* k_host,
+                                  const void* v_host, void* out_host, void* stream);
+
+/* Line-boundary step (Sec. 3.3, Eq. 5-10).  Legal only when the layer has just completed a line
+ * (visual count multiple of n, every token decoded), else LAR_ERR_BAD_STATE.
+ * While fewer than B visual tokens are cached (or on the full-cache path) it only restarts the guide
+ * queue.  Otherwise, per unit: scores the M mid tokens with the line's n*G guide queries
+ * (softmax over the mid keys, mean over queries and heads), evicts the n lowest (ties: the higher
+ * position goes first), and compacts K, V and the index map in place to
+ * [prefix | anchor | kept mid | recent], leaving an n-token buffer for the next line. */
+lar_status_t lar_line_end_score_evict(lar_cache_t* c, int layer, void* stream);
+
+/* Destroy the host object.  The slab is the caller's and is not touched. */
+lar_status_t lar_cache_destroy(lar_cache_t* c);
+
+/* Introspection for tests: synchronises `stream`, then copies to HOST buffers (each may be NULL)
+ *   lens       [batch * n_kv_heads]              live entries per unit
+ *   index_map  [batch * n_kv_heads, capacity]    original position of each slot (prefix j -> j,
+ *                                                visual token i (1-based) -> C + i - 1); -1 beyond len
+ *   scores     [batch * n_kv_heads, mid_len]     Eq. 9 scores of the last compressing line end */
+lar_status_t lar_cache_get_state(lar_cache_t* c, int layer, int32_t* lens, int32_t* index_map, float* scores,
+                                 void* stream);
+
+/* Synchronises `stream` and returns LAR_ERR_DEVICE_CHECK if any kernel recorded a failed check since
+ * the last poll (bits in *bits_out, may be NULL: 1 capacity, 2 line-end off boundary, 4 wait limit,
+ * 8 decode on an empty cache); clears the word. */
+lar_status_t lar_cache_poll_device_status(lar_cache_t* c, uint32_t* bits_out, void* stream);
+
+/* Enable (1) / disable (0) the host-side call-order checks at run time (see LAR_FLAG_NO_HOST_CHECKS). */
+lar_status_t lar_cache_set_host_checks(lar_cache_t* c, int enabled);
+
+/* Number of kernels this cache has launched so far (bookkeeping for benchmarks). */
+uint64_t lar_cache_launch_count(const lar_cache_t* c);
+
+/* The plan a cache was created with. */
+lar_status_t lar_cache_get_plan(const lar_cache_t* c, lar_plan_t* plan_out);
+
+const char* lar_status_str(lar_status_t s);
+int lar_last_cuda_error(void); /* cudaError_t of the last failed runtime call in this thread, 0 if none */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAR_H_ */

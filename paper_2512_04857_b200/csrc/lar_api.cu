@@ -1,0 +1,571 @@
+// Host side of the C ABI declared in include/lar.h: config validation, slab layout, the call-order
+// state machine and the kernel launches.  No torch types, no allocation on the hot path.
+#include "../../include/lar.h"
+
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "decode_attn.cuh"
+#include "line_end.cuh"
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+#define LAR_CUDA(call)                                   \
+    do {                                                 \
+        cudaError_t e__ = (call);                        \
+        if (e__ != cudaSuccess) {                        \
+            g_last_cuda_error = (int)e__;                \
+            (void)cudaGetLastError();                    \
+            return LAR_ERR_CUDA;                         \
+        }                                                \
+    } while (0)
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {
+    // per-cache
+    size_t off_status, off_staging;
+    // per-layer strides and the offset of layer 0
+    size_t off_state, stride_state;
+    size_t off_ptab, stride_ptab;
+    size_t off_imap, stride_imap;
+    size_t off_guide, stride_guide;
+    size_t off_scores, stride_scores;
+    size_t off_kpool, off_vpool, stride_pool;
+    size_t staging_q, staging_k, staging_v, staging_o;  // offsets inside the staging area
+    size_t total;
+};
+
+struct Derived {
+    int units, group, elt, row_bytes, cap, ppu, P, cap_pad, M, mid_pad, compressing, B, N;
+};
+
+bool derive(const lar_config_t* c, Derived& d) {
+    if (!c || c->struct_size != sizeof(lar_config_t)) return false;
+    if (c->n_layers < 1 || c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1) return false;
+    if (c->n_q_heads % c->n_kv_heads) return false;
+    d.group = c->n_q_heads / c->n_kv_heads;
+    if (!(d.group == 1 || d.group == 2 || d.group == 4 || d.group == 8)) return false;
+    if (!(c->head_dim == 64 || c->head_dim == 128)) return false;
+    if (!(c->dtype == LAR_BF16 || c->dtype == LAR_FP32)) return false;
+    if (c->cond_len < 0 || c->line_width < 1 || c->n_lines < 1 || c->anchor_len < 0) return false;
+    if (c->recent_lines < 1 || c->budget_lines < 1) return false;
+    if (c->page_tokens != 0 && c->page_tokens != 16 && c->page_tokens != 32 && c->page_tokens != 64) return false;
+    if (c->kv_splits != 0 && c->kv_splits != 1 && c->kv_splits != 2 && c->kv_splits != 4 && c->kv_splits != 8) return false;
+    if (c->warps_per_cta < 0 || c->warps_per_cta > 8 || c->stages < 0 || c->stages > 4) return false;
+    if (!(c->softmax_scale >= 0.f) || !isfinite(c->softmax_scale)) return false;
+    const long long N = (long long)c->line_width * c->n_lines;
+    if (N > (1 << 24) || (long long)c->batch * c->n_kv_heads > (1 << 24)) return false;
+    d.N = (int)N;
+    d.compressing = c->budget_lines < c->n_lines ? 1 : 0;
+    d.B = d.compressing ? c->budget_lines * c->line_width : d.N;
+    if (c->anchor_len > d.N) return false;
+    d.M = 0;
+    if (d.compressing) {
+        d.M = d.B - c->anchor_len - c->recent_lines * c->line_width;
+        if (d.M < c->line_width) return false;  // fewer than n mid candidates: not defined by the method
+    }
+    d.units = c->batch * c->n_kv_heads;
+    d.elt = c->dtype == LAR_BF16 ? 2 : 4;
+    d.row_bytes = c->head_dim * d.elt;
+    d.cap = c->cond_len + d.B;
+    d.P = c->page_tokens ? c->page_tokens : 16;
+    d.ppu = (d.cap + d.P - 1) / d.P;
+    d.cap_pad = d.ppu * d.P;
+    d.mid_pad = (int)align_up((size_t)(d.M > 0 ? d.M : 1), 4);
+    return true;
+}
+
+void make_layout(const lar_config_t* c, const Derived& d, Layout& L) {
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t Lyr = (size_t)c->n_layers, U = (size_t)d.units;
+    L.off_status = take(256);
+    const size_t qb = (size_t)c->batch * c->n_q_heads * d.row_bytes, kb = (size_t)c->batch * c->n_kv_heads * d.row_bytes;
+    L.staging_q = 0;
+    L.staging_k = align_up(qb, 256);
+    L.staging_v = L.staging_k + align_up(kb, 256);
+    L.staging_o = L.staging_v + align_up(kb, 256);
+    L.off_staging = take(L.staging_o + qb);
+    L.stride_state = align_up(U * sizeof(lar::UnitState), 256);
+    L.off_state = take(L.stride_state * Lyr);
+    L.stride_ptab = align_up(U * d.ppu * 4, 256);
+    L.off_ptab = take(L.stride_ptab * Lyr);
+    L.stride_imap = align_up(U * d.cap_pad * 4, 256);
+    L.off_imap = take(L.stride_imap * Lyr);
+    L.stride_guide = align_up(U * c->line_width * d.group * d.row_bytes, 256);
+    L.off_guide = take(L.stride_guide * Lyr);
+    L.stride_scores = align_up(U * d.mid_pad * 4, 256);
+    L.off_scores = take(L.stride_scores * Lyr);
+    L.stride_pool = align_up(U * d.ppu * d.P * d.row_bytes, 256);
+    L.off_kpool = take(L.stride_pool * Lyr);
+    L.off_vpool = take(L.stride_pool * Lyr);
+    L.total = off;
+}
+
+int pow2_floor(int x) { int p = 1; while (p * 2 <= x) p *= 2; return p; }
+
+// Launch shape of the decode kernel.  Aim: enough CTAs to cover the 148 SMs a few times, a few 16-row
+// tiles per warp at the steady-state length, all K/V of a CTA in flight at once where it fits.
+void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
+    const int tiles = (d.cap + lar::kGranule - 1) / lar::kGranule;  // tiles at the longest live length
+    int X = c->kv_splits;
+    if (X == 0) {
+        X = 1;
+        while (X < 8 && d.units * X < 592 && tiles / (X * 2) >= 4) X *= 2;
+    }
+    int W = c->warps_per_cta;
+    if (W == 0) {
+        const int per_cta = (tiles + X - 1) / X;
+        W = pow2_floor((per_cta + 2) / 3);
+        if (W < 1) W = 1;
+        if (W > 4) W = 4;
+    }
+    int NS = c->stages;
+    if (NS == 0) {
+        const int per_warp = (tiles + X * W - 1) / (X * W);
+        NS = per_warp < 3 ? (per_warp < 1 ? 1 : per_warp) : 3;
+    }
+    p.kv_splits = X;
+    p.warps_per_cta = W;
+    p.stages = NS;
+    p.decode_smem_bytes = lar::decode_smem_bytes(2 * lar::kGranule * d.row_bytes, W, NS, X, d.group, c->head_dim);
+}
+
+lar_status_t plan_query_impl(const lar_config_t* cfg, lar_plan_t* out, Derived* dout, Layout* lout) {
+    Derived d;
+    if (!cfg || !derive(cfg, d)) return LAR_ERR_INVALID_ARG;
+    Layout L;
+    make_layout(cfg, d, L);
+    lar_plan_t p;
+    memset(&p, 0, sizeof(p));
+    p.capacity = d.cap;
+    p.pages_per_unit = d.ppu;
+    p.page_tokens = d.P;
+    p.mid_len = d.M;
+    p.compressing = d.compressing;
+    choose_plan(cfg, d, p);
+    p.line_end_smem_bytes =
+        d.compressing ? lar::line_end_smem_bytes(d.row_bytes, cfg->head_dim, d.M, d.M - cfg->line_width + cfg->recent_lines * cfg->line_width, 8) : 0;
+    p.slab_bytes = L.total;
+    if (p.decode_smem_bytes > 227 * 1024 || p.line_end_smem_bytes > 227 * 1024) return LAR_ERR_INVALID_ARG;
+    if (out) *out = p;
+    if (dout) *dout = d;
+    if (lout) *lout = L;
+    return LAR_OK;
+}
+
+struct LayerShadow {
+    bool prefilled = false;
+    bool pending_decode = false;
+    int v = 0;          // live visual entries
+    int n_tok = 0;      // visual tokens appended
+    int line_fill = 0;  // tokens of the current line decoded so far
+};
+
+}  // namespace
+
+struct lar_cache {
+    lar_config_t cfg;
+    lar_plan_t plan;
+    Derived d;
+    Layout L;
+    char* slab;
+    int device;
+    bool host_checks;
+    float scale;
+    uint64_t launches;
+    int last_layer;  // layer whose cache the most recent library kernel may have written (-1 none)
+    std::vector<LayerShadow> sh;
+};
+
+namespace {
+
+lar::LayerView view_of(const lar_cache* c, int layer) {
+    lar::LayerView v;
+    const Layout& L = c->L;
+    const Derived& d = c->d;
+    v.k_pool = c->slab + L.off_kpool + L.stride_pool * layer;
+    v.v_pool = c->slab + L.off_vpool + L.stride_pool * layer;
+    v.page_table = reinterpret_cast<const int*>(c->slab + L.off_ptab + L.stride_ptab * layer);
+    v.index_map = reinterpret_cast<int*>(c->slab + L.off_imap + L.stride_imap * layer);
+    v.state = reinterpret_cast<lar::UnitState*>(c->slab + L.off_state + L.stride_state * layer);
+    v.guide = c->slab + L.off_guide + L.stride_guide * layer;
+    v.scores = reinterpret_cast<float*>(c->slab + L.off_scores + L.stride_scores * layer);
+    v.status = reinterpret_cast<unsigned*>(c->slab + L.off_status);
+    v.pages_per_unit = d.ppu;
+    v.page_tokens = d.P;
+    v.cap = d.cap;
+    v.cap_pad = d.cap_pad;
+    v.mid_pad = d.mid_pad;
+    v.cond_len = c->cfg.cond_len;
+    v.line_width = c->cfg.line_width;
+    v.budget_tokens = d.B;
+    v.anchor_len = c->cfg.anchor_len;
+    v.recent_lines = c->cfg.recent_lines;
+    v.compressing = d.compressing;
+    v.n_kv_heads = c->cfg.n_kv_heads;
+    v.group = d.group;
+    return v;
+}
+
+// ---- kernel tables ------------------------------------------------------------------------------
+using DecodeFn = void (*)(const lar::DecodeArgs);
+using LineEndFn = void (*)(const lar::LayerView, float);
+
+template <typename T, int D>
+DecodeFn decode_for_group(int G) {
+    switch (G) {
+        case 1: return lar::decode_kernel<T, D, 1>;
+        case 2: return lar::decode_kernel<T, D, 2>;
+        case 4: return lar::decode_kernel<T, D, 4>;
+        case 8: return lar::decode_kernel<T, D, 8>;
+    }
+    return nullptr;
+}
+DecodeFn decode_fn(const lar_config_t& c, int G) {
+    if (c.dtype == LAR_BF16) return c.head_dim == 64 ? decode_for_group<__nv_bfloat16, 64>(G) : decode_for_group<__nv_bfloat16, 128>(G);
+    return c.head_dim == 64 ? decode_for_group<float, 64>(G) : decode_for_group<float, 128>(G);
+}
+template <typename T, int D>
+LineEndFn line_end_for_group(int G) {
+    switch (G) {
+        case 1: return lar::line_end_kernel<T, D, 1>;
+        case 2: return lar::line_end_kernel<T, D, 2>;
+        case 4: return lar::line_end_kernel<T, D, 4>;
+        case 8: return lar::line_end_kernel<T, D, 8>;
+    }
+    return nullptr;
+}
+LineEndFn line_end_fn(const lar_config_t& c, int G) {
+    if (c.dtype == LAR_BF16) return c.head_dim == 64 ? line_end_for_group<__nv_bfloat16, 64>(G) : line_end_for_group<__nv_bfloat16, 128>(G);
+    return c.head_dim == 64 ? line_end_for_group<float, 64>(G) : line_end_for_group<float, 128>(G);
+}
+
+lar_status_t launch_append(lar_cache* c, int layer, const void* k, const void* v, int n_tokens, int is_prefix,
+                           cudaStream_t s) {
+    const lar::LayerView lv = view_of(c, layer);
+    const int U = c->d.units;
+    if (c->cfg.dtype == LAR_BF16) {
+        if (c->cfg.head_dim == 64)
+            lar::append_kernel<__nv_bfloat16, 64><<<U, 128, 0, s>>>(lv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, n_tokens, is_prefix);
+        else
+            lar::append_kernel<__nv_bfloat16, 128><<<U, 128, 0, s>>>(lv, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, n_tokens, is_prefix);
+    } else {
+        if (c->cfg.head_dim == 64)
+            lar::append_kernel<float, 64><<<U, 128, 0, s>>>(lv, (const float*)k, (const float*)v, n_tokens, is_prefix);
+        else
+            lar::append_kernel<float, 128><<<U, 128, 0, s>>>(lv, (const float*)k, (const float*)v, n_tokens, is_prefix);
+    }
+    LAR_CUDA(cudaGetLastError());
+    c->launches++;
+    c->last_layer = layer;
+    return LAR_OK;
+}
+
+lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k, const void* v, void* out, int fused,
+                           cudaStream_t s) {
+    lar::DecodeArgs a;
+    a.lv = view_of(c, layer);
+    a.q = q;
+    a.k_new = k;
+    a.v_new = v;
+    a.out = out;
+    a.scale_log2 = c->scale * 1.4426950408889634f;
+    a.fused = fused;
+    const bool pdl = (c->cfg.flags & LAR_FLAG_PDL) != 0;
+    a.prefetch = (pdl && c->last_layer != layer && c->last_layer >= 0) ? 1 : 0;
+    a.splits = c->plan.kv_splits;
+    a.stages = c->plan.stages;
+
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof(lc));
+    lc.gridDim = dim3((unsigned)(c->d.units * c->plan.kv_splits), 1, 1);
+    lc.blockDim = dim3((unsigned)(32 * c->plan.warps_per_cta), 1, 1);
+    lc.dynamicSmemBytes = (size_t)c->plan.decode_smem_bytes;
+    lc.stream = s;
+    cudaLaunchAttribute attrs[2];
+    unsigned na = 0;
+    if (c->plan.kv_splits > 1) {
+        attrs[na].id = cudaLaunchAttributeClusterDimension;
+        attrs[na].val.clusterDim.x = (unsigned)c->plan.kv_splits;
+        attrs[na].val.clusterDim.y = 1;
+        attrs[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (pdl) {
+        attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attrs[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    lc.attrs = attrs;
+    lc.numAttrs = na;
+    DecodeFn fn = decode_fn(c->cfg, c->d.group);
+    LAR_CUDA(cudaLaunchKernelEx(&lc, fn, a));
+    c->launches++;
+    c->last_layer = layer;
+    return LAR_OK;
+}
+
+bool bad_layer(const lar_cache* c, int layer) { return !c || layer < 0 || layer >= c->cfg.n_layers; }
+
+// host-side protocol: visual append
+lar_status_t check_visual_append(lar_cache* c, LayerShadow& sh) {
+    if (!c->host_checks) return LAR_OK;
+    if (!sh.prefilled && c->cfg.cond_len > 0) return LAR_ERR_BAD_STATE;
+    if (sh.pending_decode) return LAR_ERR_BAD_STATE;
+    if (sh.n_tok >= c->d.N) return LAR_ERR_CAPACITY;
+    if (sh.line_fill >= c->cfg.line_width) return LAR_ERR_CAPACITY;  // line complete: the line-end call is due
+    if (sh.v >= c->d.B) return LAR_ERR_CAPACITY;
+    return LAR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* lar_status_str(lar_status_t s) {
+    switch (s) {
+        case LAR_OK: return "ok";
+        case LAR_ERR_INVALID_ARG: return "invalid argument";
+        case LAR_ERR_BAD_STATE: return "call order violates the decode protocol";
+        case LAR_ERR_CAPACITY: return "capacity exceeded";
+        case LAR_ERR_CUDA: return "CUDA runtime error";
+        case LAR_ERR_NOMEM: return "out of memory / slab too small";
+        case LAR_ERR_DEVICE_CHECK: return "device-side check failed";
+    }
+    return "unknown status";
+}
+
+int lar_last_cuda_error(void) { return g_last_cuda_error; }
+
+lar_status_t lar_plan_query(const lar_config_t* cfg, lar_plan_t* plan_out) {
+    return plan_query_impl(cfg, plan_out, nullptr, nullptr);
+}
+
+size_t lar_cache_slab_bytes(const lar_config_t* cfg) {
+    lar_plan_t p;
+    if (plan_query_impl(cfg, &p, nullptr, nullptr) != LAR_OK) return 0;
+    return (size_t)p.slab_bytes;
+}
+
+lar_status_t lar_cache_create(const lar_config_t* cfg, void* dev_slab, size_t slab_bytes, lar_cache_t** out) {
+    if (!out) return LAR_ERR_INVALID_ARG;
+    *out = nullptr;
+    lar_plan_t plan;
+    Derived d;
+    Layout L;
+    lar_status_t st = plan_query_impl(cfg, &plan, &d, &L);
+    if (st != LAR_OK) return st;
+    if (!dev_slab || (reinterpret_cast<uintptr_t>(dev_slab) & 255u)) return LAR_ERR_INVALID_ARG;
+    if (slab_bytes < L.total) return LAR_ERR_NOMEM;
+
+    lar_cache* c = new (std::nothrow) lar_cache();
+    if (!c) return LAR_ERR_NOMEM;
+    c->cfg = *cfg;
+    c->plan = plan;
+    c->d = d;
+    c->L = L;
+    c->slab = static_cast<char*>(dev_slab);
+    c->host_checks = (cfg->flags & LAR_FLAG_NO_HOST_CHECKS) == 0;
+    c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
+    c->launches = 0;
+    c->last_layer = -1;
+    c->sh.assign((size_t)cfg->n_layers, LayerShadow());
+
+    auto fail = [&](lar_status_t e) { delete c; return e; };
+    cudaError_t ce = cudaGetDevice(&c->device);
+    if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return fail(LAR_ERR_CUDA); }
+
+    // page tables: unit u owns pages_per_unit pages of its layer's pool (identity, or shuffled)
+    const size_t per_layer = (size_t)d.units * d.ppu;
+    std::vector<int> tab(per_layer);
+    for (int layer = 0; layer < cfg->n_layers; ++layer) {
+        for (size_t i = 0; i < per_layer; ++i) tab[i] = (int)i;
+        if (cfg->flags & LAR_FLAG_SHUFFLE_PAGES) {
+            uint64_t x = 0x9E3779B97F4A7C15ull * (cfg->page_seed + 1u) + (uint64_t)layer * 0xD1B54A32D192ED03ull;
+            for (size_t i = per_layer; i > 1; --i) {
+                x ^= x >> 12; x ^= x << 25; x ^= x >> 27;
+                const size_t j = (size_t)((x * 0x2545F4914F6CDD1Dull) >> 33) % i;
+                const int t = tab[i - 1]; tab[i - 1] = tab[j]; tab[j] = t;
+            }
+        }
+        ce = cudaMemcpy(c->slab + L.off_ptab + L.stride_ptab * layer, tab.data(), per_layer * sizeof(int), cudaMemcpyHostToDevice);
+        if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; (void)cudaGetLastError(); return fail(LAR_ERR_CUDA); }
+    }
+    ce = cudaMemset(c->slab + L.off_status, 0, 256);
+    if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_state, 0, L.stride_state * cfg->n_layers);
+    if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_imap, 0xff, L.stride_imap * cfg->n_layers);
+    if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_scores, 0, L.stride_scores * cfg->n_layers);
+    if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_guide, 0, L.stride_guide * cfg->n_layers);
+    if (ce == cudaSuccess)
+        ce = cudaFuncSetAttribute((const void*)decode_fn(*cfg, d.group), cudaFuncAttributeMaxDynamicSharedMemorySize, plan.decode_smem_bytes);
+    if (ce == cudaSuccess && d.compressing)
+        ce = cudaFuncSetAttribute((const void*)line_end_fn(*cfg, d.group), cudaFuncAttributeMaxDynamicSharedMemorySize, plan.line_end_smem_bytes);
+    if (ce == cudaSuccess) ce = cudaDeviceSynchronize();
+    if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; (void)cudaGetLastError(); return fail(LAR_ERR_CUDA); }
+    *out = c;
+    return LAR_OK;
+}
+
+lar_status_t lar_cache_destroy(lar_cache_t* c) {
+    if (!c) return LAR_ERR_INVALID_ARG;
+    delete c;
+    return LAR_OK;
+}
+
+lar_status_t lar_cache_reset(lar_cache_t* c, void* stream) {
+    if (!c) return LAR_ERR_INVALID_ARG;
+    LAR_CUDA(cudaMemsetAsync(c->slab + c->L.off_state, 0, c->L.stride_state * c->cfg.n_layers, (cudaStream_t)stream));
+    for (auto& s : c->sh) s = LayerShadow();
+    c->last_layer = -1;
+    return LAR_OK;
+}
+
+lar_status_t lar_cache_set_host_checks(lar_cache_t* c, int enabled) {
+    if (!c) return LAR_ERR_INVALID_ARG;
+    c->host_checks = enabled != 0;
+    return LAR_OK;
+}
+
+uint64_t lar_cache_launch_count(const lar_cache_t* c) { return c ? c->launches : 0; }
+
+lar_status_t lar_cache_get_plan(const lar_cache_t* c, lar_plan_t* plan_out) {
+    if (!c || !plan_out) return LAR_ERR_INVALID_ARG;
+    *plan_out = c->plan;
+    return LAR_OK;
+}
+
+lar_status_t lar_append_kv(lar_cache_t* c, int layer, const void* k, const void* v, int n_tokens, void* stream) {
+    if (bad_layer(c, layer) || !k || !v || n_tokens < 1) return LAR_ERR_INVALID_ARG;
+    LayerShadow& sh = c->sh[layer];
+    const bool is_prefix = !sh.prefilled && c->cfg.cond_len > 0;
+    if (is_prefix) {
+        if (c->host_checks && n_tokens != c->cfg.cond_len) return LAR_ERR_INVALID_ARG;
+    } else {
+        if (n_tokens != 1) return LAR_ERR_INVALID_ARG;
+        lar_status_t st = check_visual_append(c, sh);
+        if (st != LAR_OK) return st;
+    }
+    lar_status_t st = launch_append(c, layer, k, v, n_tokens, is_prefix ? 1 : 0, (cudaStream_t)stream);
+    if (st != LAR_OK) return st;
+    if (is_prefix) {
+        sh.prefilled = true;
+    } else {
+        sh.pending_decode = true;
+        sh.v += 1;
+        sh.n_tok += 1;
+    }
+    return LAR_OK;
+}
+
+lar_status_t lar_decode_attn(lar_cache_t* c, int layer, const void* q, void* out, void* stream) {
+    if (bad_layer(c, layer) || !q || !out) return LAR_ERR_INVALID_ARG;
+    LayerShadow& sh = c->sh[layer];
+    if (c->host_checks && !sh.pending_decode) return LAR_ERR_BAD_STATE;
+    lar_status_t st = launch_decode(c, layer, q, nullptr, nullptr, out, 0, (cudaStream_t)stream);
+    if (st != LAR_OK) return st;
+    sh.pending_decode = false;
+    sh.line_fill += 1;
+    return LAR_OK;
+}
+
+lar_status_t lar_decode_step(lar_cache_t* c, int layer, const void* q, const void* k, const void* v, void* out,
+                             void* stream) {
+    if (bad_layer(c, layer) || !q || !k || !v || !out) return LAR_ERR_INVALID_ARG;
+    LayerShadow& sh = c->sh[layer];
+    lar_status_t st = check_visual_append(c, sh);
+    if (st != LAR_OK) return st;
+    st = launch_decode(c, layer, q, k, v, out, 1, (cudaStream_t)stream);
+    if (st != LAR_OK) return st;
+    sh.v += 1;
+    sh.n_tok += 1;
+    sh.line_fill += 1;
+    return LAR_OK;
+}
+
+lar_status_t lar_decode_step_host(lar_cache_t* c, int layer, const void* q_host, const void* k_host, const void* v_host,
+                                  void* out_host, void* stream) {
+    if (bad_layer(c, layer) || !q_host || !k_host || !v_host || !out_host) return LAR_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t qb = (size_t)c->cfg.batch * c->cfg.n_q_heads * c->d.row_bytes;
+    const size_t kb = (size_t)c->cfg.batch * c->cfg.n_kv_heads * c->d.row_bytes;
+    char* stg = c->slab + c->L.off_staging;
+    LAR_CUDA(cudaMemcpyAsync(stg + c->L.staging_q, q_host, qb, cudaMemcpyHostToDevice, s));
+    LAR_CUDA(cudaMemcpyAsync(stg + c->L.staging_k, k_host, kb, cudaMemcpyHostToDevice, s));
+    LAR_CUDA(cudaMemcpyAsync(stg + c->L.staging_v, v_host, kb, cudaMemcpyHostToDevice, s));
+    const int saved = c->last_layer;
+    c->last_layer = layer;  // a copy precedes the kernel: never prefetch ahead of it
+    lar_status_t st = lar_decode_step(c, layer, stg + c->L.staging_q, stg + c->L.staging_k, stg + c->L.staging_v,
+                                      stg + c->L.staging_o, stream);
+    if (st != LAR_OK) { c->last_layer = saved; return st; }
+    LAR_CUDA(cudaMemcpyAsync(out_host, stg + c->L.staging_o, qb, cudaMemcpyDeviceToHost, s));
+    return LAR_OK;
+}
+
+lar_status_t lar_line_end_score_evict(lar_cache_t* c, int layer, void* stream) {
+    if (bad_layer(c, layer)) return LAR_ERR_INVALID_ARG;
+    LayerShadow& sh = c->sh[layer];
+    if (c->host_checks) {
+        if (sh.pending_decode || sh.line_fill != c->cfg.line_width) return LAR_ERR_BAD_STATE;
+    }
+    if (c->d.compressing) {
+        const lar::LayerView lv = view_of(c, layer);
+        LineEndFn fn = line_end_fn(c->cfg, c->d.group);
+        fn<<<c->d.units, 256, c->plan.line_end_smem_bytes, (cudaStream_t)stream>>>(lv, c->scale * 1.4426950408889634f);
+        LAR_CUDA(cudaGetLastError());
+        c->launches++;
+        c->last_layer = layer;
+        if (sh.v >= c->d.B) sh.v -= c->cfg.line_width;
+    }
+    sh.line_fill = 0;
+    return LAR_OK;
+}
+
+lar_status_t lar_cache_get_state(lar_cache_t* c, int layer, int32_t* lens, int32_t* index_map, float* scores,
+                                 void* stream) {
+    if (bad_layer(c, layer)) return LAR_ERR_INVALID_ARG;
+    LAR_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    const int U = c->d.units;
+    std::vector<lar::UnitState> st((size_t)U);
+    LAR_CUDA(cudaMemcpy(st.data(), c->slab + c->L.off_state + c->L.stride_state * layer, (size_t)U * sizeof(lar::UnitState),
+                        cudaMemcpyDeviceToHost));
+    if (lens)
+        for (int u = 0; u < U; ++u) lens[u] = st[u].len;
+    if (index_map) {
+        std::vector<int> raw((size_t)U * c->d.cap_pad);
+        LAR_CUDA(cudaMemcpy(raw.data(), c->slab + c->L.off_imap + c->L.stride_imap * layer, raw.size() * sizeof(int),
+                            cudaMemcpyDeviceToHost));
+        for (int u = 0; u < U; ++u)
+            for (int s = 0; s < c->d.cap; ++s)
+                index_map[(size_t)u * c->d.cap + s] = s < st[u].len ? raw[(size_t)u * c->d.cap_pad + s] : -1;
+    }
+    if (scores && c->d.M > 0) {
+        std::vector<float> raw((size_t)U * c->d.mid_pad);
+        LAR_CUDA(cudaMemcpy(raw.data(), c->slab + c->L.off_scores + c->L.stride_scores * layer, raw.size() * sizeof(float),
+                            cudaMemcpyDeviceToHost));
+        for (int u = 0; u < U; ++u)
+            memcpy(scores + (size_t)u * c->d.M, raw.data() + (size_t)u * c->d.mid_pad, (size_t)c->d.M * sizeof(float));
+    }
+    return LAR_OK;
+}
+
+lar_status_t lar_cache_poll_device_status(lar_cache_t* c, uint32_t* bits_out, void* stream) {
+    if (!c) return LAR_ERR_INVALID_ARG;
+    LAR_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    unsigned bits = 0;
+    LAR_CUDA(cudaMemcpy(&bits, c->slab + c->L.off_status, sizeof(bits), cudaMemcpyDeviceToHost));
+    if (bits) LAR_CUDA(cudaMemset(c->slab + c->L.off_status, 0, sizeof(bits)));
+    if (bits_out) *bits_out = bits;
+    return bits ? LAR_ERR_DEVICE_CHECK : LAR_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,113 @@
+"""CPU-only checks of the C ABI: the library loads, exports every declared symbol, and the host-side
+logic (config validation, derived plan, slab sizing, argument checks) behaves as documented."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2512_04857_b200 import lar, workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(lar_[a-z0-9_]+)\s*\(", text))
+    return names
+
+
+def test_library_loads_and_exports_every_declared_symbol():
+    L = lar.lib()
+    names = _declared_symbols()
+    assert {"lar_cache_create", "lar_append_kv", "lar_decode_attn", "lar_line_end_score_evict",
+            "lar_cache_destroy"} <= names
+    for n in sorted(names):
+        assert hasattr(L, n), f"liblar.so does not export {n}"
+
+
+def test_status_strings():
+    L = lar.lib()
+    assert L.lar_status_str(0) == b"ok"
+    assert len({L.lar_status_str(i) for i in range(7)}) == 7
+
+
+@pytest.mark.parametrize("name", list(W.WORKLOADS))
+def test_plan_of_each_workload(name):
+    w = W.WORKLOADS[name]
+    p = lar.lar_plan_query(lar.config_from_workload(w))
+    assert p.capacity == w.cond_len + w.budget_tokens
+    assert p.mid_len == w.mid_len and p.compressing == 1
+    assert p.pages_per_unit * p.page_tokens >= p.capacity
+    assert p.kv_splits in (1, 2, 4, 8) and 1 <= p.warps_per_cta <= 8 and 1 <= p.stages <= 4
+    assert p.decode_smem_bytes <= 227 * 1024 and p.line_end_smem_bytes <= 227 * 1024
+    kv = 2 * w.n_layers * w.n_units * p.pages_per_unit * p.page_tokens * w.head_dim * w.elt_bytes
+    assert kv <= p.slab_bytes <= kv * 1.3 + (1 << 22)
+    assert lar.lar_cache_slab_bytes(lar.config_from_workload(w)) == p.slab_bytes
+    pf = lar.lar_plan_query(lar.config_from_workload(w.full_cache()))
+    assert pf.compressing == 0 and pf.mid_len == 0 and pf.capacity == w.cond_len + w.n_visual
+
+
+def _cfg(**kw):
+    base = dict(n_layers=1, batch=1, n_q_heads=4, n_kv_heads=4, head_dim=64, dtype="bf16", cond_len=4,
+                line_width=8, n_lines=8, anchor_len=8, recent_lines=1, budget_lines=4)
+    base.update(kw)
+    return lar.make_config(**base)
+
+
+@pytest.mark.parametrize("bad", [
+    dict(n_q_heads=6, n_kv_heads=4),          # Hq % Hkv != 0
+    dict(n_q_heads=12, n_kv_heads=4),         # group 3
+    dict(head_dim=96),
+    dict(dtype=7),
+    dict(recent_lines=0),
+    dict(budget_lines=2),                     # B - N_init - r n = 0 < n
+    dict(anchor_len=17, budget_lines=4),      # mid would be 7 < n
+    dict(page_tokens=24),
+    dict(kv_splits=3),
+    dict(warps_per_cta=9),
+    dict(stages=5),
+    dict(n_layers=0),
+    dict(cond_len=-1),
+    dict(softmax_scale=-1.0),
+])
+def test_invalid_configs_are_rejected(bad):
+    cfg = _cfg(**bad)
+    plan = lar.lar_plan_t()
+    assert lar.lib().lar_plan_query(C.byref(cfg), C.byref(plan)) == lar.LAR_ERR_INVALID_ARG
+    assert lar.lar_cache_slab_bytes(cfg) == 0
+
+
+def test_struct_size_is_checked_and_null_arguments():
+    L = lar.lib()
+    cfg = _cfg()
+    cfg.struct_size = 8
+    assert L.lar_plan_query(C.byref(cfg), None) == lar.LAR_ERR_INVALID_ARG
+    assert L.lar_plan_query(None, None) == lar.LAR_ERR_INVALID_ARG
+    cfg = _cfg()
+    assert L.lar_plan_query(C.byref(cfg), None) == lar.LAR_OK
+    out = C.c_void_p()
+    # no slab / misaligned slab / too small: rejected before any CUDA work
+    assert L.lar_cache_create(C.byref(cfg), None, 1 << 30, C.byref(out)) == lar.LAR_ERR_INVALID_ARG
+    assert L.lar_cache_create(C.byref(cfg), 4096 + 8, 1 << 30, C.byref(out)) == lar.LAR_ERR_INVALID_ARG
+    assert L.lar_cache_create(C.byref(cfg), 4096, 16, C.byref(out)) == lar.LAR_ERR_NOMEM
+    assert L.lar_cache_create(C.byref(cfg), 4096, 1 << 30, None) == lar.LAR_ERR_INVALID_ARG
+    for fn, args in [(L.lar_cache_destroy, (None,)), (L.lar_cache_reset, (None, None)),
+                     (L.lar_append_kv, (None, 0, None, None, 1, None)),
+                     (L.lar_decode_attn, (None, 0, None, None, None)),
+                     (L.lar_line_end_score_evict, (None, 0, None))]:
+        assert fn(*args) == lar.LAR_ERR_INVALID_ARG
+    assert L.lar_cache_launch_count(None) == 0
+
+
+def test_full_cache_budget_and_overrides():
+    p = lar.lar_plan_query(_cfg(budget_lines=8))
+    assert p.compressing == 0 and p.capacity == 4 + 64
+    p = lar.lar_plan_query(_cfg(budget_lines=100))
+    assert p.compressing == 0 and p.capacity == 4 + 64
+    p = lar.lar_plan_query(_cfg(kv_splits=4, warps_per_cta=8, stages=2, page_tokens=32))
+    assert (p.kv_splits, p.warps_per_cta, p.stages, p.page_tokens) == (4, 8, 2, 32)

@@ -1,0 +1,130 @@
+"""GPU parity: CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
+
+Bars: attention outputs max-abs 1e-4 (fp32) / 2e-2 (bf16); kept-token positions bit-exact, except
+near-ties within 1e-5 relative of the eviction boundary, which are counted."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2512_04857_b200 import lar, workloads as W
+from _harness import TOL, pick_units, run_parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(rep, w, allow_near_ties=0):
+    assert not rep.mismatches, rep.mismatches
+    assert rep.max_abs_err <= TOL[w.dtype], rep.max_abs_err
+    assert rep.near_ties <= allow_near_ties, rep.near_ties
+    assert rep.outputs_compared > 0
+
+
+# ------------------------------------------------------------------ the tiny fp32 configs, every unit
+@pytest.mark.parametrize("name", ["tiny", "tiny_b"])
+@pytest.mark.parametrize("fused", [True, False])
+def test_tiny_configs_all_units(name, fused):
+    w = W.WORKLOADS[name]
+    rep = run_parity(w, fused=fused)
+    _check(rep, w)
+    assert rep.compressions == 8 * (w.n_lines - w.budget_lines)
+    assert rep.max_score_rel_err < 1e-4
+
+
+def test_tiny_full_cache_path():
+    w = W.WORKLOADS["tiny"].full_cache()
+    rep = run_parity(w)
+    _check(rep, w)
+    assert rep.compressions == 0
+
+
+@pytest.mark.parametrize("splits,warps,stages", [(1, 1, 1), (1, 8, 3), (2, 2, 2), (4, 1, 4), (8, 4, 1), (8, 8, 2)])
+def test_launch_shapes(splits, warps, stages):
+    w = W.WORKLOADS["tiny_b"]
+    rep = run_parity(w, cfg_overrides=dict(kv_splits=splits, warps_per_cta=warps, stages=stages))
+    _check(rep, w)
+
+
+@pytest.mark.parametrize("page_tokens", [16, 32, 64])
+def test_shuffled_pages(page_tokens):
+    w = W.WORKLOADS["tiny_b"]
+    rep = run_parity(w, cfg_overrides=dict(page_tokens=page_tokens, flags=lar.LAR_FLAG_SHUFFLE_PAGES, page_seed=7))
+    _check(rep, w)
+
+
+def test_pdl_flag_multi_layer():
+    w = W.WORKLOADS["tiny_b"].scaled(n_layers=3)
+    rep = run_parity(w, cfg_overrides=dict(flags=lar.LAR_FLAG_PDL))
+    _check(rep, w)
+
+
+# ------------------------------------------------------------------ scaled-down shapes of the paper's models
+SMALL = {
+    "llamagen": W.WORKLOADS["llamagen_xl"].scaled(n_layers=2, batch=2, n_q_heads=4, n_kv_heads=4),
+    "janus": W.WORKLOADS["janus_pro_7b"].scaled(n_layers=2, batch=2, n_q_heads=4, n_kv_heads=4),
+    "lumina": W.WORKLOADS["lumina_768"].scaled(n_layers=1, batch=1, n_q_heads=4, n_kv_heads=4, n_lines=16),
+    "gqa": W.WORKLOADS["gqa_1024"].scaled(n_layers=1, batch=2, n_q_heads=8, n_kv_heads=2, n_lines=14),
+}
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_small_bf16_shapes_all_units(name):
+    w = SMALL[name]
+    rep = run_parity(w)
+    _check(rep, w, allow_near_ties=2)
+    assert rep.compressions > 0
+
+
+# ------------------------------------------------------------------ edge cases
+@pytest.mark.parametrize("kw", [
+    dict(cond_len=0),                                        # no prefix
+    dict(anchor_len=0),                                      # no anchor
+    dict(anchor_len=5, recent_lines=2, budget_lines=5),      # anchor not a whole line
+    dict(n_q_heads=8, n_kv_heads=4),                         # G = 2
+    dict(n_q_heads=8, n_kv_heads=1),                         # G = 8
+    dict(head_dim=128),                                      # fp32, 512-byte rows
+    dict(line_width=7, n_lines=9, anchor_len=7, recent_lines=1, budget_lines=3, cond_len=3),  # odd sizes
+    dict(line_width=1, n_lines=40, anchor_len=1, recent_lines=2, budget_lines=6),             # 1-token lines
+    dict(dtype="bf16", head_dim=64, n_q_heads=4, n_kv_heads=2),
+])
+def test_edge_shapes(kw):
+    w = W.WORKLOADS["tiny_b"].scaled(**kw)
+    rep = run_parity(w)
+    _check(rep, w, allow_near_ties=1)
+
+
+def test_partial_generation_stops_mid_line():
+    w = W.WORKLOADS["tiny_b"]
+    rep = run_parity(w, n_steps=w.line_width * 9 + 5)
+    _check(rep, w)
+
+
+# ------------------------------------------------------------------ full-size shapes, sampled units
+FULL = [("llamagen_xl", 2, 6), ("janus_pro_7b", 2, 6), ("lumina_768", 1, 4), ("gqa_1024", 1, 4)]
+
+
+@pytest.mark.parametrize("name,layers,n_units", FULL)
+def test_full_size_shapes_sampled_units(name, layers, n_units):
+    """Full batch / heads / grid / budget of the benchmark shapes in the launch configuration the
+    benchmark times (fused step, default plan, PDL); fewer layers (layers are independent and
+    identically shaped), oracle on a sample of units."""
+    w = W.WORKLOADS[name].scaled(n_layers=layers)
+    rep = run_parity(w, units=pick_units(w, n_units, seed=1), gen_device="cuda",
+                     cfg_overrides=dict(flags=lar.LAR_FLAG_PDL))
+    _check(rep, w, allow_near_ties=2)
+    assert rep.compressions == n_units * (w.n_lines - w.budget_lines)
+
+
+@pytest.mark.parametrize("name,steps", [("janus_pro_7b", None), ("gqa_1024", 65 * 20)])
+def test_full_cache_path_full_size_sampled(name, steps):
+    w = W.WORKLOADS[name].scaled(n_layers=1).full_cache()
+    rep = run_parity(w, units=pick_units(w, 3, seed=2), gen_device="cuda", n_steps=steps)
+    _check(rep, w)
+
+
+def test_generator_gpu_matches_cpu():
+    w = W.WORKLOADS["janus_pro_7b"].scaled(batch=2)
+    a = W.gen_tokens(w, 1, 10, 14, "cpu")
+    b = W.gen_tokens(w, 1, 10, 14, "cuda")
+    for x, y in zip(a, b):
+        diff = (x.float() != y.float().cpu()).float().mean().item()
+        assert diff < 1e-4

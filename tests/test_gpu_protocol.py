@@ -1,0 +1,140 @@
+"""GPU tests of the call protocol, error reporting and the host-buffer entry point."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2512_04857_b200 import lar, workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _small(**kw):
+    base = dict(n_layers=2, batch=2, n_q_heads=4, n_kv_heads=4, head_dim=64, dtype="bf16", cond_len=4,
+                line_width=8, n_lines=8, anchor_len=8, recent_lines=1, budget_lines=4)
+    base.update(kw)
+    return lar.make_config(**base)
+
+
+def _bufs(cfg, dev="cuda:0"):
+    dt = torch.bfloat16 if cfg.dtype == lar.LAR_BF16 else torch.float32
+    g = torch.Generator(device="cpu").manual_seed(1)
+    mk = lambda *s: torch.randn(*s, generator=g).to(dt).to(dev)
+    return dict(q=mk(cfg.batch, cfg.n_q_heads, cfg.head_dim), k=mk(cfg.batch, cfg.n_kv_heads, cfg.head_dim),
+                v=mk(cfg.batch, cfg.n_kv_heads, cfg.head_dim),
+                kc=mk(cfg.batch, cfg.n_kv_heads, max(cfg.cond_len, 1), cfg.head_dim),
+                vc=mk(cfg.batch, cfg.n_kv_heads, max(cfg.cond_len, 1), cfg.head_dim),
+                out=torch.zeros(cfg.batch, cfg.n_q_heads, cfg.head_dim, dtype=dt, device=dev))
+
+
+def _status(fn, *a):
+    try:
+        fn(*a)
+        return lar.LAR_OK
+    except lar.LarError as e:
+        return e.status
+
+
+def test_call_order_errors():
+    cfg = _small()
+    c = lar.Cache(cfg)
+    b = _bufs(cfg)
+    # visual append before the prefill, decode without an append, wrong prefix length
+    assert _status(c.decode_step, 0, b["q"], b["k"], b["v"], b["out"]) == lar.LAR_ERR_BAD_STATE
+    assert _status(c.decode_attn, 0, b["q"], b["out"]) == lar.LAR_ERR_BAD_STATE
+    assert _status(c.append_kv, 0, b["kc"], b["vc"], 3) == lar.LAR_ERR_INVALID_ARG
+    c.append_kv(0, b["kc"], b["vc"], 4)
+    assert _status(c.append_kv, 0, b["k"], b["v"], 2) == lar.LAR_ERR_INVALID_ARG
+    assert _status(c.line_end_score_evict, 0) == lar.LAR_ERR_BAD_STATE       # no line finished
+    c.append_kv(0, b["k"], b["v"], 1)
+    assert _status(c.append_kv, 0, b["k"], b["v"], 1) == lar.LAR_ERR_BAD_STATE   # decode is due
+    assert _status(c.line_end_score_evict, 0) == lar.LAR_ERR_BAD_STATE
+    c.decode_attn(0, b["q"], b["out"])
+    assert _status(c.decode_attn, 0, b["q"], b["out"]) == lar.LAR_ERR_BAD_STATE
+    for _ in range(7):
+        c.decode_step(0, b["q"], b["k"], b["v"], b["out"])
+    # the line is complete: the n-token buffer is exhausted until the line-end call
+    assert _status(c.decode_step, 0, b["q"], b["k"], b["v"], b["out"]) == lar.LAR_ERR_CAPACITY
+    c.line_end_score_evict(0)
+    c.decode_step(0, b["q"], b["k"], b["v"], b["out"])
+    assert _status(c.decode_step, 5, b["q"], b["k"], b["v"], b["out"]) == lar.LAR_ERR_INVALID_ARG
+    assert _status(c.decode_step, 0, None, b["k"], b["v"], b["out"]) == lar.LAR_ERR_INVALID_ARG
+    assert c.poll_device_status() == 0
+    # layers are independent: layer 1 still needs its prefill
+    assert _status(c.decode_step, 1, b["q"], b["k"], b["v"], b["out"]) == lar.LAR_ERR_BAD_STATE
+    lens, imap = c.get_state(0)
+    assert (lens == 4 + 9).all() and (imap[:, :13] == np.arange(13)).all() and (imap[:, 13:] == -1).all()
+    c.reset()
+    lens, _ = c.get_state(0)
+    assert (lens == 0).all()
+    assert c.launch_count() > 0
+    c.close()
+
+
+def test_device_side_checks_record_status_instead_of_faulting():
+    cfg = _small(flags=lar.LAR_FLAG_NO_HOST_CHECKS)
+    c = lar.Cache(cfg)
+    b = _bufs(cfg)
+    c.append_kv(0, b["kc"], b["vc"], 4)
+    for _ in range(3):
+        c.decode_step(0, b["q"], b["k"], b["v"], b["out"])
+    c.line_end_score_evict(0)                       # off a line boundary -> recorded, nothing touched
+    assert c.poll_device_status() & 2
+    lens, _ = c.get_state(0)
+    assert (lens == 7).all()
+    for _ in range(29):                             # fill to capacity C + B = 36 without line ends
+        c.decode_step(0, b["q"], b["k"], b["v"], b["out"])
+    assert c.poll_device_status() == 0
+    c.decode_step(0, b["q"], b["k"], b["v"], b["out"])   # one more: no room, row is not stored
+    assert c.poll_device_status() & 1
+    lens, _ = c.get_state(0)
+    assert (lens == 36).all()
+    assert torch.isfinite(b["out"].float()).all()
+    assert c.poll_device_status() == 0              # polling clears the word
+    c.close()
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    cfg = _small(n_layers=1)
+    b = _bufs(cfg)
+    outs = []
+    for host in (False, True):
+        c = lar.Cache(cfg)
+        c.append_kv(0, b["kc"], b["vc"], 4)
+        if host:
+            pin = {k: b[k].cpu().pin_memory() for k in ("q", "k", "v")}
+            out = torch.zeros_like(b["out"], device="cpu").pin_memory()
+        res = []
+        for i in range(8):
+            if host:
+                c.decode_step_host(0, pin["q"], pin["k"], pin["v"], out)
+                torch.cuda.synchronize()
+                res.append(out.clone())
+            else:
+                c.decode_step(0, b["q"], b["k"], b["v"], b["out"])
+                torch.cuda.synchronize()
+                res.append(b["out"].cpu().clone())
+        outs.append(torch.stack(res))
+        assert c.poll_device_status() == 0
+        c.close()
+    assert torch.equal(outs[0], outs[1])
+
+
+def test_softmax_scale_override_and_single_row_cache():
+    # C = 0 and the very first token: attention over one entry returns v exactly
+    cfg = _small(n_layers=1, cond_len=0, softmax_scale=0.37, dtype="fp32")
+    c = lar.Cache(cfg)
+    b = _bufs(cfg)
+    c.decode_step(0, b["q"], b["k"], b["v"], b["out"])
+    torch.cuda.synchronize()
+    assert torch.allclose(b["out"], b["v"], atol=1e-6)
+    # second token: two-entry softmax with the overridden scale
+    k2, v2 = b["k"] * 0.5, b["v"] + 1.0
+    c.decode_step(0, b["q"], k2, v2, b["out"])
+    torch.cuda.synchronize()
+    logit = torch.stack([(b["q"] * b["k"]).sum(-1), (b["q"] * k2).sum(-1)], -1).double() * 0.37
+    p = torch.softmax(logit, -1)
+    ref = p[..., :1] * b["v"].double() + p[..., 1:] * v2.double()
+    assert torch.allclose(b["out"].double(), ref, atol=1e-5)
+    c.close()
