@@ -191,15 +191,6 @@ class Runner:
         self.graphs = None
         self.launches_per_generation = 0
 
-    def _enqueue_line(self, line, with_line_end=True):
-        w, c = self.w, self.cache
-        if line == 0:
-            c.reset()
-            if w.cond_len:
-                for layer in range(w.n_layers):
-                    c.append_kv(layer, self.kc[layer], self.vc[layer], w.cond_len)
-        return self._enqueue_decode(line), (self._enqueue_line_end(line) if with_line_end else 0)
-
     def _enqueue_decode(self, line):
         w, c = self.w, self.cache
         for t in range(w.line_width):
@@ -245,6 +236,20 @@ class Runner:
         """Replay one whole image generation on the current stream; optionally record (start, end) events
         around the decode part of every line."""
         torch = self.torch
+        if self.graphs is None:            # eager mode
+            for line in range(self.w.n_lines):
+                if line == 0:
+                    self.cache.reset()
+                    if self.w.cond_len:
+                        for layer in range(self.w.n_layers):
+                            self.cache.append_kv(layer, self.kc[layer], self.vc[layer], self.w.cond_len)
+                if events is not None:
+                    events[line][0].record()
+                self._enqueue_decode(line)
+                if events is not None:
+                    events[line][1].record()
+                self._enqueue_line_end(line)
+            return
         for line, (ga, gb) in enumerate(self.graphs):
             if events is not None:
                 e0, e1 = events[line]
@@ -255,10 +260,6 @@ class Runner:
                 ga.replay()
             if gb is not None:
                 gb.replay()
-
-    def eager_generation(self):
-        for line in range(self.w.n_lines):
-            self._enqueue_line(line)
 
     def close(self):
         self.graphs = None
@@ -370,10 +371,16 @@ def run_ours(args):
     torch.cuda.set_device(dev)
     peak, peak_kind = load_peaks()
     w = W.WORKLOADS[args.workload]
+    if args.layers:
+        w = w.scaled(n_layers=args.layers)
 
     def bench_workload(wl, steps, warmup, sample_clocks):
         r = Runner(wl, dev, args)
-        r.capture()
+        if args.eager:
+            r.launches_per_generation = (wl.n_layers * (wl.n_visual + (1 if wl.cond_len else 0))
+                                         + (0 if wl.is_full_cache else wl.n_layers * (wl.n_lines - 1)))
+        else:
+            r.capture()
         sampler = ClockSampler(local) if sample_clocks else None
         total_ms, decode_ms, clocks, halves = time_generations(r, steps, warmup, dist, sampler)
         bits = r.cache.poll_device_status()
@@ -475,6 +482,8 @@ def main():
     ap.add_argument("--warps", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--page-tokens", type=int, default=0)
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling / small cases)")
+    ap.add_argument("--eager", action="store_true", help="plain stream launches instead of CUDA graphs (profiling)")
     ap.add_argument("--no-pdl", action="store_true")
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

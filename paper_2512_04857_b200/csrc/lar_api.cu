@@ -12,6 +12,7 @@
 
 #include "common.cuh"
 #include "decode_attn.cuh"
+#include "decode_mma.cuh"
 #include "line_end.cuh"
 
 namespace {
@@ -120,24 +121,21 @@ void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
     int X = c->kv_splits;
     if (X == 0) {
         X = 1;
-        while (X < 8 && d.units * X < 592 && tiles / (X * 2) >= 4) X *= 2;
+        while (X < 8 && d.units * X < 740 && tiles / (X * 2) >= 2) X *= 2;
     }
     int W = c->warps_per_cta;
-    if (W == 0) {
-        const int per_cta = (tiles + X - 1) / X;
-        W = pow2_floor((per_cta + 2) / 3);
-        if (W < 1) W = 1;
-        if (W > 4) W = 4;
-    }
+    if (W == 0) W = 2;
     int NS = c->stages;
     if (NS == 0) {
         const int per_warp = (tiles + X * W - 1) / (X * W);
-        NS = per_warp < 3 ? (per_warp < 1 ? 1 : per_warp) : 3;
+        NS = per_warp < 2 ? 1 : 2;
     }
     p.kv_splits = X;
     p.warps_per_cta = W;
     p.stages = NS;
-    p.decode_smem_bytes = lar::decode_smem_bytes(2 * lar::kGranule * d.row_bytes, W, NS, X, d.group, c->head_dim);
+    p.decode_smem_bytes = c->dtype == LAR_BF16
+                              ? lar::decode_mma_smem_bytes(c->head_dim, W, NS, X, d.group)
+                              : lar::decode_smem_bytes(2 * lar::kGranule * d.row_bytes, W, NS, X, d.group, c->head_dim);
 }
 
 lar_status_t plan_query_impl(const lar_config_t* cfg, lar_plan_t* out, Derived* dout, Layout* lout) {
@@ -184,6 +182,8 @@ struct lar_cache {
     float scale;
     uint64_t launches;
     int last_layer;  // layer whose cache the most recent library kernel may have written (-1 none)
+    lar::TensorMaps tmaps;  // bf16 only
+    int rows_per_layer;     // pool rows between consecutive layers
     std::vector<LayerShadow> sh;
 };
 
@@ -217,7 +217,57 @@ lar::LayerView view_of(const lar_cache* c, int layer) {
     return v;
 }
 
+// ---- tensor maps (bf16 decode path) -----------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+lar_status_t make_tensor_maps(lar_cache* c) {
+    void* fp = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t ce = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fp, cudaEnableDefault, &qres);
+    if (ce != cudaSuccess || !fp || qres != cudaDriverEntryPointSuccess) {
+        g_last_cuda_error = (int)(ce != cudaSuccess ? ce : cudaErrorUnknown);
+        (void)cudaGetLastError();
+        return LAR_ERR_CUDA;
+    }
+    EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fp);
+    c->rows_per_layer = (int)(c->L.stride_pool / (size_t)c->d.row_bytes);
+    const cuuint64_t gdim[2] = {(cuuint64_t)c->cfg.head_dim, (cuuint64_t)c->rows_per_layer * (cuuint64_t)c->cfg.n_layers};
+    const cuuint64_t gstride[1] = {(cuuint64_t)c->d.row_bytes};
+    const cuuint32_t estr[2] = {1, 1};
+    for (int h = 0; h < 4; ++h) {
+        const cuuint32_t box[2] = {64, (cuuint32_t)(4 * (h + 1))};
+        for (int kv = 0; kv < 2; ++kv) {
+            CUtensorMap* m = kv == 0 ? &c->tmaps.k[h] : &c->tmaps.v[h];
+            void* base = c->slab + (kv == 0 ? c->L.off_kpool : c->L.off_vpool);
+            CUresult r = encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) {
+                g_last_cuda_error = (int)cudaErrorInvalidValue;
+                return LAR_ERR_CUDA;
+            }
+        }
+    }
+    return LAR_OK;
+}
+
 // ---- kernel tables ------------------------------------------------------------------------------
+using DecodeMmaFn = void (*)(const lar::DecodeArgs, const lar::TensorMaps, const int);
+template <int D>
+DecodeMmaFn decode_mma_for_group(int G) {
+    switch (G) {
+        case 1: return lar::decode_mma_kernel<D, 1>;
+        case 2: return lar::decode_mma_kernel<D, 2>;
+        case 4: return lar::decode_mma_kernel<D, 4>;
+        case 8: return lar::decode_mma_kernel<D, 8>;
+    }
+    return nullptr;
+}
+DecodeMmaFn decode_mma_fn(const lar_config_t& c, int G) {
+    return c.head_dim == 64 ? decode_mma_for_group<64>(G) : decode_mma_for_group<128>(G);
+}
 using DecodeFn = void (*)(const lar::DecodeArgs);
 using LineEndFn = void (*)(const lar::LayerView, float);
 
@@ -232,7 +282,6 @@ DecodeFn decode_for_group(int G) {
     return nullptr;
 }
 DecodeFn decode_fn(const lar_config_t& c, int G) {
-    if (c.dtype == LAR_BF16) return c.head_dim == 64 ? decode_for_group<__nv_bfloat16, 64>(G) : decode_for_group<__nv_bfloat16, 128>(G);
     return c.head_dim == 64 ? decode_for_group<float, 64>(G) : decode_for_group<float, 128>(G);
 }
 template <typename T, int D>
@@ -308,8 +357,13 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
     }
     lc.attrs = attrs;
     lc.numAttrs = na;
-    DecodeFn fn = decode_fn(c->cfg, c->d.group);
-    LAR_CUDA(cudaLaunchKernelEx(&lc, fn, a));
+    if (c->cfg.dtype == LAR_BF16) {
+        DecodeMmaFn fn = decode_mma_fn(c->cfg, c->d.group);
+        LAR_CUDA(cudaLaunchKernelEx(&lc, fn, a, c->tmaps, layer * c->rows_per_layer));
+    } else {
+        DecodeFn fn = decode_fn(c->cfg, c->d.group);
+        LAR_CUDA(cudaLaunchKernelEx(&lc, fn, a));
+    }
     c->launches++;
     c->last_layer = layer;
     return LAR_OK;
@@ -406,12 +460,20 @@ lar_status_t lar_cache_create(const lar_config_t* cfg, void* dev_slab, size_t sl
     if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_imap, 0xff, L.stride_imap * cfg->n_layers);
     if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_scores, 0, L.stride_scores * cfg->n_layers);
     if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_guide, 0, L.stride_guide * cfg->n_layers);
+    // rows of a page beyond the live length are read by short tiles with weight 0: they must be finite
+    if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_kpool, 0, L.stride_pool * cfg->n_layers);
+    if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_vpool, 0, L.stride_pool * cfg->n_layers);
     if (ce == cudaSuccess)
-        ce = cudaFuncSetAttribute((const void*)decode_fn(*cfg, d.group), cudaFuncAttributeMaxDynamicSharedMemorySize, plan.decode_smem_bytes);
+        ce = cudaFuncSetAttribute(cfg->dtype == LAR_BF16 ? (const void*)decode_mma_fn(*cfg, d.group) : (const void*)decode_fn(*cfg, d.group),
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, plan.decode_smem_bytes);
     if (ce == cudaSuccess && d.compressing)
         ce = cudaFuncSetAttribute((const void*)line_end_fn(*cfg, d.group), cudaFuncAttributeMaxDynamicSharedMemorySize, plan.line_end_smem_bytes);
     if (ce == cudaSuccess) ce = cudaDeviceSynchronize();
     if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; (void)cudaGetLastError(); return fail(LAR_ERR_CUDA); }
+    if (cfg->dtype == LAR_BF16) {
+        lar_status_t ts = make_tensor_maps(c);
+        if (ts != LAR_OK) return fail(ts);
+    }
     *out = c;
     return LAR_OK;
 }
