@@ -77,10 +77,13 @@ typedef struct lar_config {
     float softmax_scale;   /* 0 selects 1/sqrt(head_dim) (Eq. 2) */
     int32_t page_tokens;   /* tokens per physical page: 16, 32 or 64; 0 selects 16 */
     uint32_t flags;        /* LAR_FLAG_* */
-    int32_t kv_splits;     /* CTAs (one thread-block cluster) per unit in decode: 0 auto, else 1,2,4,8 */
-    int32_t warps_per_cta; /* decode warps per CTA: 0 auto, else 1..8 */
-    int32_t stages;        /* 16-row K/V stages in flight per warp: 0 auto, else 1..4 */
+    int32_t kv_splits;     /* fp32 only: CTAs (one thread-block cluster) per unit in decode: 0 auto, else 1,2,4,8 */
+    int32_t warps_per_cta; /* decode warps: bf16 consumer warps per CTA, 0 auto, else 1..4;
+                              fp32 warps per CTA, 0 auto, else 1..8 */
+    int32_t stages;        /* 16-row K/V stages: bf16 depth of the CTA's ring, 0 auto, else 2..32;
+                              fp32 stages in flight per warp, 0 auto, else 1..4 */
     uint32_t page_seed;    /* seed of LAR_FLAG_SHUFFLE_PAGES */
+    int32_t decode_ctas;   /* bf16 only: CTAs of the persistent decode grid: 0 selects 148 (one per SM), else 1..1024 */
 } lar_config_t;
 
 /* What lar_cache_create derived from a config (introspection; also usable without a GPU). */
@@ -94,6 +97,9 @@ typedef struct lar_plan {
     int32_t line_end_smem_bytes;
     int32_t compressing;    /* 1 if budget_lines < n_lines */
     uint64_t slab_bytes;
+    int32_t decode_ctas;    /* CTAs per decode launch */
+    int32_t max_segments;   /* bf16: most CTAs one unit's rows are spread over (scratch partials per unit) */
+    uint64_t scratch_bytes; /* part of the slab used as decode scratch (partials, tickets) */
 } lar_plan_t;
 
 /* Validate a config and report the derived plan.  No CUDA call is made.
@@ -104,7 +110,9 @@ lar_status_t lar_plan_query(const lar_config_t* cfg, lar_plan_t* plan_out);
 
 /* Bytes of device memory the caller must provide for a cache of this config (0 if invalid).
  * The slab holds the paged K/V pools of all layers, page tables, per-unit lengths, the slot ->
- * original-position index maps, the guide queues (Eq. 8) and the last score vectors (Eq. 9). */
+ * original-position index maps, the guide queues (Eq. 8), the last score vectors (Eq. 9) and the
+ * decode scratch (partial results of units whose rows are spread over several CTAs).
+ * The scratch is shared by all layers: calls on one cache must be ordered on one stream. */
 size_t lar_cache_slab_bytes(const lar_config_t* cfg);
 
 /* Create a cache over a caller-allocated device slab (256-byte aligned, >= lar_cache_slab_bytes).
@@ -124,12 +132,13 @@ lar_status_t lar_append_kv(lar_cache_t* c, int layer, const void* k, const void*
 
 /* Decode attention (Eq. 2-3) of the token appended last: out = softmax(q K^T scale) V over every live
  * entry of the unit (prefix + retained visual tokens + the new token), per query head.
- * q, out: device, [batch, n_q_heads, head_dim].  Also stores q in the layer's guide queue (Eq. 8).
+ * q, out: device, [batch, n_q_heads, head_dim], 16-byte aligned.  Also stores q in the layer's guide
+ * queue (Eq. 8).
  * LAR_ERR_BAD_STATE unless a visual token was appended to this layer since its last decode. */
 lar_status_t lar_decode_attn(lar_cache_t* c, int layer, const void* q, void* out, void* stream);
 
 /* lar_append_kv(n_tokens = 1) + lar_decode_attn fused into one kernel launch (Eq. 4 then Eq. 2).
- * k, v: device, [batch, n_kv_heads, head_dim]. */
+ * k, v: device, [batch, n_kv_heads, head_dim], 16-byte aligned. */
 lar_status_t lar_decode_step(lar_cache_t* c, int layer, const void* q, const void* k, const void* v,
                              void* out, void* stream);
 

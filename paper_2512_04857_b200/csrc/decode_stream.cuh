@@ -1,0 +1,611 @@
+// bf16 decode attention (Eq. 2-3) as one persistent, warp-specialised streaming kernel per layer-step,
+// fused with the append of the step's token (Eq. 4) and the guide-queue push (Eq. 8).
+//
+// Work decomposition.  The live rows of every unit = (sequence, KV head) are cut into 16-row tiles;
+// all tiles of the layer form one list (unit-major) that is dealt out in equal contiguous ranges
+// to the CTAs of the grid (one CTA per SM), so every SM streams the same number of bytes whatever
+// the number of units.  The part of a unit that falls into one CTA is a *segment*.  A unit that lies
+// inside one CTA is finished there; a unit cut by a range boundary leaves one partial (m, l, o) per
+// segment in a global scratch area and the CTA that delivers the last partial (an atomic ticket, no
+// waiting) merges them.
+//
+// Inside a CTA three roles run concurrently, coupled only by mbarriers (every wait is bounded):
+//   warp 0           producer: walks the CTA's tile range and keeps a ring of NS stages filled with
+//                    K and V tiles (cp.async.bulk.tensor, 2-D tiled, 128-byte swizzle); also fetches
+//                    the queries (and the step's new k, v row) of each segment into a small ring.
+//   warps 1 .. W     consumers: tile j of the range goes to consumer j % W:
+//                        S = Q K^T     mma.sync m16n8k16 (bf16 in, fp32 out), rows = the G heads
+//                        online softmax in fp32 (base-2, scale folded into the logits)
+//                        O += P V      same instruction, V fragments via ldmatrix.trans
+//                    and at the end of a segment each consumer leaves its partial in shared memory.
+//   warp W + 1       epilogue: merges the W partials of a segment with the step's own token,
+//                    writes the output row (or the scratch partial + ticket), stores the new K/V
+//                    row, the index-map entry and the guide-queue row.
+// The producer never waits for arithmetic, so the HBM stream is continuous across unit boundaries.
+// With programmatic dependent launch the producer fills its ring with tiles of this layer's cache
+// while the preceding kernel (another layer) is still running; everything else waits for it.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace lar {
+
+struct TensorMaps {
+    CUtensorMap k[4];  // box heights 4, 8, 12, 16 rows over the K pools of all layers
+    CUtensorMap v[4];
+};
+
+struct StreamArgs {
+    LayerView lv;
+    const void* q;      // [units * G][d]
+    const void* k_new;  // [units][d]   (fused only)
+    const void* v_new;
+    void* out;          // [units * G][d]
+    float* partials;    // scratch [units][max_seg][G][d + 2]
+    int* tickets;       // scratch [units], zero between launches
+    int* done;          // scratch, one counter, zero between launches
+    float scale_log2;   // softmax scale * log2(e)
+    int fused;          // 1: the step's token comes from k_new / v_new and is appended by this kernel
+    int prefetch;       // 1: cached K/V may be fetched before the preceding kernel has finished
+    int n_units, n_stages, max_seg;
+    int pool_row_base;  // first pool row of this layer in the tensor maps
+};
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&t);
+}
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
+
+template <int D>
+struct MmaTraits {
+    static constexpr int ROW_BYTES = D * 2;
+    static constexpr int HALVES = D / 64;             // 128-byte column blocks per row
+    static constexpr int SUB_BYTES = kGranule * 128;  // one [16][64] swizzled block
+    static constexpr int TILE_BYTES = HALVES * SUB_BYTES;
+    static constexpr int STAGE_BYTES = 2 * TILE_BYTES;  // K tile + V tile
+    static constexpr int KSTEPS = D / 16;
+    static constexpr int NTILES = D / 8;
+};
+
+// byte offset of 16-byte chunk `c` of row `r` inside a tile stored as HALVES swizzled [16][128 B] blocks
+template <int D>
+__device__ __forceinline__ uint32_t tile_off(int r, int c) {
+    return (uint32_t)((c >> 3) * MmaTraits<D>::SUB_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+
+// ---- shared-memory plan of decode_stream_kernel (host and device agree through these) -------------
+__host__ __device__ constexpr int stream_q_slots(int G) { return G <= 2 ? 8 : 4; }
+__host__ __device__ constexpr int stream_q_entry_bytes(int D, int G) { return ((G + 2) * D * 2 + 127) / 128 * 128; }
+__host__ __device__ constexpr int stream_fixed_smem_bytes(int D, int G, int W) {
+    return 1024                                               // slack: the ring starts on a 1024-byte boundary
+           + stream_q_slots(G) * stream_q_entry_bytes(D, G)   // query ring
+           + 2 * (W + 1) * G * (D + 2) * 4                    // two partial buffers
+           + (2 * stream_q_slots(G) + 4) * 8 + 16;            // query / partial barriers, abort flag
+}
+__host__ __device__ constexpr int stream_smem_bytes(int D, int G, int W, int NS) {
+    return stream_fixed_smem_bytes(D, G, W) + NS * (2 * (D / 64) * kGranule * 128 + 16);  // stage + its 2 barriers
+}
+
+// Wait on an mbarrier phase; gives up (and raises the CTA-wide abort flag) after ~1 s of SM clocks or as
+// soon as another role has given up, so that no role can hang.
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    unsigned spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 15u) == 0u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > 2000000000LL) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ float exp2_or_zero(float m_part, float m_all) {
+    return m_part == -INFINITY ? 0.f : exp2f(m_part - m_all);
+}
+
+// CTA that owns tile t of a list of `total` tiles dealt to P <= total CTAs as ranges [p total / P, (p + 1) total / P)
+__device__ __forceinline__ int range_owner(long long t, long long total, int P) {
+    return (int)(((t + 1) * P - 1) / total);
+}
+
+template <int D, int G>
+__global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs a, const __grid_constant__ TensorMaps tm) {
+    using TR = MmaTraits<D>;
+    using T16 = __nv_bfloat16;
+    constexpr int NQ = stream_q_slots(G);
+    constexpr int QENT = stream_q_entry_bytes(D, G);
+    constexpr int PS = D + 2;  // floats per (warp, head) partial: o[D], m, l
+    constexpr int PER = D / 32;
+    extern __shared__ unsigned char smem_raw[];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int W = (int)(blockDim.x >> 5) - 2;  // consumer warps
+    const int NS = a.n_stages;
+    const int P = (int)gridDim.x, p = (int)blockIdx.x;
+    const LayerView& lv = a.lv;
+
+    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* smem = smem_raw + (ring - smem_u32(smem_raw));
+    unsigned char* qring_ptr = smem + (size_t)NS * TR::STAGE_BYTES;
+    const uint32_t qring = smem_u32(qring_ptr);
+    float* pbuf = reinterpret_cast<float*>(qring_ptr + NQ * QENT);
+    const int pbuf_floats = (W + 1) * G * PS;
+    unsigned char* bars_ptr = reinterpret_cast<unsigned char*>(pbuf + 2 * pbuf_floats);
+    const uint32_t bars = smem_u32(bars_ptr);
+    const uint32_t bar_full = bars, bar_empty = bars + NS * 8;
+    const uint32_t bar_qfull = bars + 2 * NS * 8, bar_qempty = bar_qfull + NQ * 8;
+    const uint32_t bar_pfull = bar_qempty + NQ * 8, bar_pempty = bar_pfull + 2 * 8;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_ptr + (2 * NS + 2 * NQ + 4) * 8);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(bar_full + s * 8, 1);
+            mbar_init(bar_empty + s * 8, 1);
+        }
+        for (int s = 0; s < NQ; ++s) {
+            mbar_init(bar_qfull + s * 8, 1);
+            mbar_init(bar_qempty + s * 8, (uint32_t)(W + 1));
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar_pfull + s * 8, (uint32_t)W);
+            mbar_init(bar_pempty + s * 8, 1);
+        }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    if (!a.prefetch) grid_dep_wait();
+
+    // ---- the layer's tile list and this CTA's range of it (units decode in lock-step: one length)
+    const int len = __ldcg(&lv.state[0].len);
+    const int n_tok = __ldcg(&lv.state[0].n_tok);
+    const int T = len > 0 ? (len + kGranule - 1) / kGranule : 1;  // an empty cache is one tile of 0 rows
+    const long long total = (long long)a.n_units * T;
+    const int Pe = total < P ? (int)total : P;  // CTAs that get tiles: every range is non-empty
+    const long long t_begin = p < Pe ? (long long)p * total / Pe : 0, t_end = p < Pe ? (long long)(p + 1) * total / Pe : 0;
+    const int n_tiles = (int)(t_end - t_begin);
+    const int u0 = (int)(t_begin / T);
+    const int n_segs = n_tiles > 0 ? (int)((t_end - 1) / T) - u0 + 1 : 0;
+
+    if (warp == 0) {
+        // =========================================================================== producer
+        bool dep_waited = !a.prefetch;
+        bool ok = true;
+        int q_next = 0;  // next segment whose inputs have not been requested yet (lane 0)
+        const int fill_end = n_tiles < NS ? n_tiles : NS;
+
+        auto describe = [&](int jj, int& y, int& rows, int& tile) {
+            const long long t = t_begin + jj;
+            const int unit = (int)(t / T);
+            tile = (int)(t - (long long)unit * T);
+            const int row0 = tile * kGranule;
+            rows = len - row0 < kGranule ? len - row0 : kGranule;
+            if (rows > 0) {
+                const int page = __ldg(&lv.page_table[unit * lv.pages_per_unit + row0 / lv.page_tokens]);
+                y = a.pool_row_base + page * lv.page_tokens + row0 % lv.page_tokens;
+            } else {
+                y = 0;
+            }
+        };
+        auto issue_inputs = [&](int seg) -> bool {  // lane 0: q (and the step's k, v) of segment `seg`
+            const int slot = seg % NQ;
+            if (seg >= NQ && !wait_or_abort(bar_qempty + slot * 8, (uint32_t)((seg / NQ - 1) & 1), abort_flag)) return false;
+            const int unit = u0 + seg;
+            const bool closes = (long long)(unit + 1) * T <= t_end;  // the segment holds the unit's last tile
+            const bool with_kv = a.fused && closes;
+            const uint32_t bar = bar_qfull + slot * 8, dst = qring + slot * QENT;
+            mbar_expect_tx(bar, (uint32_t)((G + (with_kv ? 2 : 0)) * D * 2));
+            bulk_g2s(dst, reinterpret_cast<const T16*>(a.q) + (size_t)unit * G * D, G * D * 2, bar);
+            if (with_kv) {
+                bulk_g2s(dst + G * D * 2, reinterpret_cast<const T16*>(a.k_new) + (size_t)unit * D, D * 2, bar);
+                bulk_g2s(dst + (G + 1) * D * 2, reinterpret_cast<const T16*>(a.v_new) + (size_t)unit * D, D * 2, bar);
+            }
+            return true;
+        };
+
+        int y_n = 0, rows_n = 0, tile_n = 0;
+        if (lane < n_tiles) describe(lane, y_n, rows_n, tile_n);
+        for (int j0 = 0; j0 < n_tiles && ok; j0 += 32) {
+            const int y = y_n, rows = rows_n, tile = tile_n;
+            if (j0 + 32 + lane < n_tiles) describe(j0 + 32 + lane, y_n, rows_n, tile_n);  // next batch: hides the table reads
+            const int cnt = n_tiles - j0 < 32 ? n_tiles - j0 : 32;
+            for (int i = 0; i < cnt; ++i) {
+                const int j = j0 + i;
+                const int yi = __shfl_sync(0xffffffffu, y, i), ri = __shfl_sync(0xffffffffu, rows, i);
+                const int ti = __shfl_sync(0xffffffffu, tile, i);
+                if (lane == 0) {
+                    if (dep_waited && (j == 0 || ti == 0)) ok = issue_inputs(q_next++);
+                    const int s = j % NS;
+                    if (ok && j >= NS) ok = wait_or_abort(bar_empty + s * 8, (uint32_t)((j / NS - 1) & 1), abort_flag);
+                    if (ok) {
+                        const uint32_t bar = bar_full + s * 8, dst = ring + (uint32_t)s * TR::STAGE_BYTES;
+                        if (ri > 0) {
+                            const int hsel = (ri + 3) / 4 - 1;  // box of 4 * (hsel + 1) rows
+                            mbar_expect_tx(bar, (uint32_t)(2 * 4 * (hsel + 1) * TR::ROW_BYTES));
+#pragma unroll
+                            for (int h = 0; h < TR::HALVES; ++h) {
+                                tma_load_2d(dst + h * TR::SUB_BYTES, &tm.k[hsel], h * 64, yi, bar);
+                                tma_load_2d(dst + TR::TILE_BYTES + h * TR::SUB_BYTES, &tm.v[hsel], h * 64, yi, bar);
+                            }
+                        } else {
+                            mbar_arrive(bar);  // nothing to fetch: release the consumer
+                        }
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) break;
+                if (!dep_waited && j == fill_end - 1) {
+                    // the ring is full of this layer's cache; everything else depends on the preceding kernel
+                    grid_dep_wait();
+                    grid_dep_launch();
+                    dep_waited = true;
+                    if (lane == 0) {
+                        const int seg_now = (int)((t_begin + j) / T) - u0;
+                        while (ok && q_next <= seg_now) ok = issue_inputs(q_next++);
+                    }
+                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                    if (!ok) break;
+                }
+            }
+        }
+        if (!dep_waited) {
+            grid_dep_wait();
+            grid_dep_launch();
+        }
+        if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
+    } else if (warp <= W) {
+        // =========================================================================== consumers
+        grid_dep_wait();
+        grid_dep_launch();
+        const int cw = warp - 1;
+        const int quad = lane & 3, qrow = lane >> 2;  // fragment coordinates
+        bool ok = true;
+        for (int seg = 0; seg < n_segs && ok; ++seg) {
+            const int unit = u0 + seg;
+            const long long ub = (long long)unit * T;
+            const int jb = (int)((ub > t_begin ? ub : t_begin) - t_begin);
+            const int je = (int)((ub + T < t_end ? ub + T : t_end) - t_begin);
+
+            // ---- Q fragments (A operand): row qrow = head, 16 columns per k-step; heads >= G are zero rows
+            const int qs = seg % NQ;
+            ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag);
+            if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+            uint32_t qa0[TR::KSTEPS], qa2[TR::KSTEPS];
+            {
+                const unsigned char* Qs = qring_ptr + qs * QENT;
+#pragma unroll
+                for (int s = 0; s < TR::KSTEPS; ++s) {
+                    qa0[s] = 0u;
+                    qa2[s] = 0u;
+                    if (qrow < G) {
+                        qa0[s] = *reinterpret_cast<const uint32_t*>(Qs + (qrow * D + 16 * s + 2 * quad) * 2);
+                        qa2[s] = *reinterpret_cast<const uint32_t*>(Qs + (qrow * D + 16 * s + 8 + 2 * quad) * 2);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_qempty + qs * 8);
+
+            float m = -INFINITY, l = 0.f;  // head qrow; l is this thread's share of the row sum
+            float o[TR::NTILES][4];
+#pragma unroll
+            for (int t = 0; t < TR::NTILES; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
+
+            for (int j = jb + ((cw - jb % W) + W) % W; j < je; j += W) {
+                const int s = j % NS;
+                ok = wait_or_abort(bar_full + s * 8, (uint32_t)((j / NS) & 1), abort_flag);
+                if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+                const int tile = (int)(t_begin + j - ub);
+                const int rows = len - tile * kGranule < kGranule ? len - tile * kGranule : kGranule;
+                const uint32_t Ks = ring + (uint32_t)s * TR::STAGE_BYTES;
+                const uint32_t Vs = Ks + TR::TILE_BYTES;
+                if (rows > 0) {
+                    // S[head][key] for the 16 keys of the tile: two n-tiles of 8 keys
+                    float sc[2][4];
+#pragma unroll
+                    for (int jn = 0; jn < 2; ++jn) {
+                        sc[jn][0] = sc[jn][1] = sc[jn][2] = sc[jn][3] = 0.f;
+#pragma unroll
+                        for (int i = 0; i < TR::KSTEPS / 2; ++i) {
+                            uint32_t b[4];
+                            ldmatrix_x4(Ks + tile_off<D>(8 * jn + (lane & 7), 4 * i + (lane >> 3)), b);
+                            mma_bf16(sc[jn], qa0[2 * i], 0u, qa2[2 * i], 0u, b[0], b[1]);
+                            mma_bf16(sc[jn], qa0[2 * i + 1], 0u, qa2[2 * i + 1], 0u, b[2], b[3]);
+                        }
+                    }
+                    // online softmax over the keys this thread holds: 2*quad, 2*quad+1 (+8)
+                    float sv[4];
+#pragma unroll
+                    for (int jn = 0; jn < 2; ++jn) {
+                        sv[2 * jn + 0] = (8 * jn + 2 * quad + 0 < rows) ? sc[jn][0] * a.scale_log2 : -INFINITY;
+                        sv[2 * jn + 1] = (8 * jn + 2 * quad + 1 < rows) ? sc[jn][1] * a.scale_log2 : -INFINITY;
+                    }
+                    float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                    const float m_new = fmaxf(m, mx);
+                    const float corr = exp2f(m - m_new);
+                    float pr[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) pr[i] = exp2f(sv[i] - m_new);
+                    l = l * corr + (pr[0] + pr[1]) + (pr[2] + pr[3]);
+                    m = m_new;
+                    if (__any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+                        for (int t = 0; t < TR::NTILES; ++t) { o[t][0] *= corr; o[t][1] *= corr; }
+                    }
+                    const uint32_t pa0 = pack_bf16(pr[0], pr[1]), pa2 = pack_bf16(pr[2], pr[3]);
+                    // a short box leaves rows of the V tile unwritten: their weight is 0, but 0 * (stale NaN) is not
+                    const int box_rows = (rows + 3) & ~3;
+                    if (box_rows < kGranule) {
+                        const int n16 = (kGranule - box_rows) * 8;  // 16-byte chunks per 128-byte-wide block
+                        for (int i = lane; i < n16 * TR::HALVES; i += 32) {
+                            const int h = i / n16, c = i - h * n16;
+                            asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(Vs + h * TR::SUB_BYTES + box_rows * 128 + c * 16), "r"(0u) : "memory");
+                        }
+                        __syncwarp();
+                    }
+                    // O[head][d] += P V
+#pragma unroll
+                    for (int t = 0; t < TR::NTILES / 2; ++t) {
+                        uint32_t b[4];
+                        ldmatrix_x4_trans(Vs + tile_off<D>((lane & 7) + 8 * ((lane >> 3) & 1), 2 * t + (lane >> 4)), b);
+                        mma_bf16(o[2 * t], pa0, 0u, pa2, 0u, b[0], b[1]);
+                        mma_bf16(o[2 * t + 1], pa0, 0u, pa2, 0u, b[2], b[3]);
+                    }
+                    if (box_rows < kGranule) fence_proxy_async_smem();  // zero-fill before the next TMA write
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_empty + s * 8);
+            }
+            if (!ok) break;
+
+            // ---- this warp's partial of the segment -> shared memory
+            const int buf = seg & 1;
+            if (seg >= 2) {
+                ok = wait_or_abort(bar_pempty + buf * 8, (uint32_t)((seg / 2 - 1) & 1), abort_flag);
+                if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+            }
+            l += __shfl_xor_sync(0xffffffffu, l, 1);
+            l += __shfl_xor_sync(0xffffffffu, l, 2);
+            if (qrow < G) {
+                float* dstp = pbuf + buf * pbuf_floats + (cw * G + qrow) * PS;
+#pragma unroll
+                for (int t = 0; t < TR::NTILES; ++t)
+                    *reinterpret_cast<float2*>(dstp + 8 * t + 2 * quad) = make_float2(o[t][0], o[t][1]);
+                if (quad == 0) {
+                    dstp[D] = m;
+                    dstp[D + 1] = l;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_pfull + buf * 8);
+        }
+        if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
+    } else {
+        // =========================================================================== epilogue
+        grid_dep_wait();
+        grid_dep_launch();
+        bool ok = true;
+        T16* outp = reinterpret_cast<T16*>(a.out);
+        for (int seg = 0; seg < n_segs && ok; ++seg) {
+            const int unit = u0 + seg;
+            const long long ub = (long long)unit * T;
+            const bool opens = ub >= t_begin, closes = ub + T <= t_end;
+            const int qs = seg % NQ, buf = seg & 1;
+            ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag);
+            if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+            const unsigned char* Qs = qring_ptr + qs * QENT;
+            const uint16_t* Q16 = reinterpret_cast<const uint16_t*>(Qs);
+
+            // ---- the token of this step (Eq. 4, 8): logit per head, value row, stores
+            float s_new[G], v_new[PER];
+            const bool with_new = a.fused && closes;
+#pragma unroll
+            for (int g = 0; g < G; ++g) s_new[g] = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < PER; ++i) v_new[i] = 0.f;
+            if (closes) {
+                if (with_new) {
+                    const uint16_t* K16 = Q16 + G * D;
+                    const uint16_t* V16 = K16 + D;
+                    float kf[PER];
+#pragma unroll
+                    for (int i = 0; i < PER; ++i) {
+                        kf[i] = bf16_bits_to_float(K16[lane + 32 * i]);
+                        v_new[i] = bf16_bits_to_float(V16[lane + 32 * i]);
+                    }
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        float sv = 0.f;
+#pragma unroll
+                        for (int i = 0; i < PER; ++i) sv = fmaf(bf16_bits_to_float(Q16[g * D + lane + 32 * i]), kf[i], sv);
+#pragma unroll
+                        for (int off = 16; off >= 1; off >>= 1) sv += __shfl_xor_sync(0xffffffffu, sv, off);
+                        s_new[g] = sv * a.scale_log2;
+                    }
+                    if (len < lv.cap) {
+                        const size_t off = row_offset(lv, unit, len, TR::ROW_BYTES);
+                        const uint32_t* K32 = reinterpret_cast<const uint32_t*>(K16);
+                        const uint32_t* V32 = reinterpret_cast<const uint32_t*>(V16);
+                        for (int i = lane; i < D / 2; i += 32) {
+                            reinterpret_cast<uint32_t*>(lv.k_pool + off)[i] = K32[i];
+                            reinterpret_cast<uint32_t*>(lv.v_pool + off)[i] = V32[i];
+                        }
+                        if (lane == 0) lv.index_map[(size_t)unit * lv.cap_pad + len] = lv.cond_len + n_tok;
+                    } else if (lane == 0) {
+                        atomicOr(lv.status, kStCapacity);
+                    }
+                } else if (!a.fused && len == 0 && lane == 0) {
+                    atomicOr(lv.status, kStEmpty);
+                }
+                // Eq. 8: the queries join the guide queue of the line being generated
+                const int tok = a.fused ? n_tok : n_tok - 1;  // 0-based visual index of this step's token
+                if (tok >= 0) {
+                    const int slot = tok % lv.line_width;
+                    uint32_t* gq = reinterpret_cast<uint32_t*>(reinterpret_cast<T16*>(lv.guide) +
+                                                               (((size_t)unit * lv.line_width + slot) * G) * D);
+                    const uint32_t* Q32 = reinterpret_cast<const uint32_t*>(Qs);
+                    for (int i = lane; i < G * D / 2; i += 32) gq[i] = Q32[i];
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_qempty + qs * 8);
+
+            // ---- merge the consumers' partials (+ the step's token)
+            ok = wait_or_abort(bar_pfull + buf * 8, (uint32_t)((seg / 2) & 1), abort_flag);
+            if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+            const float* pb = pbuf + buf * pbuf_floats;
+            float Mg[G], Lg[G], Og[G][PER];
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                float M = s_new[g];
+                for (int w = 0; w < W; ++w) M = fmaxf(M, pb[(w * G + g) * PS + D]);
+                const float f_new = exp2_or_zero(s_new[g], M);
+                float L = f_new;
+#pragma unroll
+                for (int i = 0; i < PER; ++i) Og[g][i] = v_new[i] * f_new;
+                for (int w = 0; w < W; ++w) {
+                    const float* pw = pb + (w * G + g) * PS;
+                    const float f = exp2_or_zero(pw[D], M);
+                    if (f != 0.f) {
+                        L = fmaf(pw[D + 1], f, L);
+#pragma unroll
+                        for (int i = 0; i < PER; ++i) Og[g][i] = fmaf(pw[lane + 32 * i], f, Og[g][i]);
+                    }
+                }
+                Mg[g] = M;
+                Lg[g] = L;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_pempty + buf * 8);
+
+            if (opens && closes) {
+                // the whole unit lies in this CTA
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const float inv = Lg[g] > 0.f ? 1.f / Lg[g] : 0.f;
+#pragma unroll
+                    for (int i = 0; i < PER; ++i)
+                        outp[((size_t)unit * G + g) * D + lane + 32 * i] = __float2bfloat16_rn(Og[g][i] * inv);
+                }
+            } else {
+                // the unit is shared with neighbouring CTAs: leave a partial, the last one to arrive merges
+                const int p_first = range_owner(ub, total, Pe);
+                const int n_parts = range_owner(ub + T - 1, total, Pe) - p_first + 1;
+                if (n_parts > a.max_seg) {  // cannot happen with the host's sizing of the scratch area
+                    if (lane == 0) atomicOr(lv.status, kStCapacity);
+                    continue;
+                }
+                float* mine = a.partials + ((size_t)unit * a.max_seg + (p - p_first)) * G * PS;
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+#pragma unroll
+                    for (int i = 0; i < PER; ++i) mine[g * PS + lane + 32 * i] = Og[g][i];
+                    if (lane == 0) {
+                        mine[g * PS + D] = Mg[g];
+                        mine[g * PS + D + 1] = Lg[g];
+                    }
+                }
+                __threadfence();
+                __syncwarp();
+                int ticket = 0;
+                if (lane == 0) ticket = atomicAdd(a.tickets + unit, 1);
+                ticket = __shfl_sync(0xffffffffu, ticket, 0);
+                if (ticket == n_parts - 1) {
+                    __threadfence();
+                    const float* all = a.partials + (size_t)unit * a.max_seg * G * PS;
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        float M = -INFINITY;
+                        for (int s = 0; s < n_parts; ++s) M = fmaxf(M, __ldcg(all + (s * G + g) * PS + D));
+                        float L = 0.f, O[PER];
+#pragma unroll
+                        for (int i = 0; i < PER; ++i) O[i] = 0.f;
+                        for (int s = 0; s < n_parts; ++s) {
+                            const float* ps = all + (s * G + g) * PS;
+                            const float f = exp2_or_zero(__ldcg(ps + D), M);
+                            if (f != 0.f) {
+                                L = fmaf(__ldcg(ps + D + 1), f, L);
+#pragma unroll
+                                for (int i = 0; i < PER; ++i) O[i] = fmaf(__ldcg(ps + lane + 32 * i), f, O[i]);
+                            }
+                        }
+                        const float inv = L > 0.f ? 1.f / L : 0.f;
+#pragma unroll
+                        for (int i = 0; i < PER; ++i)
+                            outp[((size_t)unit * G + g) * D + lane + 32 * i] = __float2bfloat16_rn(O[i] * inv);
+                    }
+                    if (lane == 0) a.tickets[unit] = 0;
+                }
+            }
+        }
+        if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
+
+        // ---- the CTA that finishes last advances the lengths (nobody reads them any more in this launch)
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) {
+            __threadfence();
+            last = atomicAdd(a.done, 1) == P - 1 ? 1 : 0;
+        }
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+            if (a.fused) {
+                UnitState ns;
+                ns.len = len < lv.cap ? len + 1 : len;
+                ns.n_tok = n_tok + 1;
+                for (int u = lane; u < a.n_units; u += 32) lv.state[u] = ns;
+            }
+            if (lane == 0) *a.done = 0;
+        }
+    }
+
+    // ---- a role gave up: let the copies still in flight land before the shared memory is released
+    __syncthreads();
+    if (*abort_flag && threadIdx.x == 0) {
+        for (int s = 0; s < NS && s < n_tiles; ++s) {
+            const int j_last = s + (n_tiles - 1 - s) / NS * NS;  // last tile that may have been sent to stage s
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar_full + s * 8, (uint32_t)((j_last / NS) & 1)) && clock64() - t0 < 200000000LL) {}
+        }
+    }
+}
+
+}  // namespace lar

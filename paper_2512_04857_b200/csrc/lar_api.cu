@@ -12,7 +12,7 @@
 
 #include "common.cuh"
 #include "decode_attn.cuh"
-#include "decode_mma.cuh"
+#include "decode_stream.cuh"
 #include "line_end.cuh"
 
 namespace {
@@ -41,13 +41,17 @@ struct Layout {
     size_t off_guide, stride_guide;
     size_t off_scores, stride_scores;
     size_t off_kpool, off_vpool, stride_pool;
+    size_t off_partials, off_tickets, tickets_bytes;  // decode scratch (shared by the layers)
     size_t staging_q, staging_k, staging_v, staging_o;  // offsets inside the staging area
     size_t total;
 };
 
 struct Derived {
     int units, group, elt, row_bytes, cap, ppu, P, cap_pad, M, mid_pad, compressing, B, N;
+    int ctas, max_seg;  // bf16 decode: CTAs of the persistent grid, most segments one unit is cut into
 };
+
+constexpr int kDefaultDecodeCtas = 148;  // one per SM of a B200
 
 bool derive(const lar_config_t* c, Derived& d) {
     if (!c || c->struct_size != sizeof(lar_config_t)) return false;
@@ -61,7 +65,12 @@ bool derive(const lar_config_t* c, Derived& d) {
     if (c->recent_lines < 1 || c->budget_lines < 1) return false;
     if (c->page_tokens != 0 && c->page_tokens != 16 && c->page_tokens != 32 && c->page_tokens != 64) return false;
     if (c->kv_splits != 0 && c->kv_splits != 1 && c->kv_splits != 2 && c->kv_splits != 4 && c->kv_splits != 8) return false;
-    if (c->warps_per_cta < 0 || c->warps_per_cta > 8 || c->stages < 0 || c->stages > 4) return false;
+    if (c->dtype == LAR_BF16) {
+        if (c->warps_per_cta < 0 || c->warps_per_cta > 4 || c->stages < 0 || c->stages == 1 || c->stages > 32) return false;
+    } else {
+        if (c->warps_per_cta < 0 || c->warps_per_cta > 8 || c->stages < 0 || c->stages > 4) return false;
+    }
+    if (c->decode_ctas < 0 || c->decode_ctas > 1024) return false;
     if (!(c->softmax_scale >= 0.f) || !isfinite(c->softmax_scale)) return false;
     const long long N = (long long)c->line_width * c->n_lines;
     if (N > (1 << 24) || (long long)c->batch * c->n_kv_heads > (1 << 24)) return false;
@@ -82,6 +91,17 @@ bool derive(const lar_config_t* c, Derived& d) {
     d.ppu = (d.cap + d.P - 1) / d.P;
     d.cap_pad = d.ppu * d.P;
     d.mid_pad = (int)align_up((size_t)(d.M > 0 ? d.M : 1), 4);
+    // A unit of T tiles is cut into at most ceil(T / floor(U T / P)) + 1 segments (never more than T or P).
+    d.ctas = c->decode_ctas ? c->decode_ctas : kDefaultDecodeCtas;
+    d.max_seg = 1;
+    const int t_max = (d.cap + lar::kGranule - 1) / lar::kGranule;
+    for (int T = 1; T <= t_max; ++T) {
+        const long long chunk = (long long)d.units * T / d.ctas;
+        long long b = chunk >= 1 ? (T + chunk - 1) / chunk + 1 : T;
+        if (b > T) b = T;
+        if (b > d.ctas) b = d.ctas;
+        if (b > d.max_seg) d.max_seg = (int)b;
+    }
     return true;
 }
 
@@ -109,14 +129,38 @@ void make_layout(const lar_config_t* c, const Derived& d, Layout& L) {
     L.stride_pool = align_up(U * d.ppu * d.P * d.row_bytes, 256);
     L.off_kpool = take(L.stride_pool * Lyr);
     L.off_vpool = take(L.stride_pool * Lyr);
+    L.off_partials = take(c->dtype == LAR_BF16 ? U * d.max_seg * d.group * (c->head_dim + 2) * sizeof(float) : 0);
+    L.tickets_bytes = (U + 1) * sizeof(int);  // one ticket per unit + the CTA counter
+    L.off_tickets = take(L.tickets_bytes);
     L.total = off;
 }
 
-int pow2_floor(int x) { int p = 1; while (p * 2 <= x) p *= 2; return p; }
 
-// Launch shape of the decode kernel.  Aim: enough CTAs to cover the 148 SMs a few times, a few 16-row
-// tiles per warp at the steady-state length, all K/V of a CTA in flight at once where it fits.
+// Launch shape of the decode kernel.
+// bf16: persistent streaming kernel, one CTA per SM, W consumer warps and a ring of NS 16-row K/V stages;
+// a CTA stays below half of the SM's shared memory so that the next layer's kernel can move in and fill
+// its ring while this one is still streaming (programmatic dependent launch).
+// fp32: one cluster of X CTAs per unit, W warps per CTA, NS stages per warp.
 void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
+    if (c->dtype == LAR_BF16) {
+        const int W = c->warps_per_cta ? c->warps_per_cta : 4;
+        int NS = c->stages;
+        if (NS == 0) {
+            const int budget = 110 * 1024;
+            const int stage = 2 * (c->head_dim / 64) * lar::kGranule * 128 + 16;
+            const int fixed = c->head_dim == 64 ? lar::stream_fixed_smem_bytes(64, d.group, W) : lar::stream_fixed_smem_bytes(128, d.group, W);
+            NS = (budget - fixed) / stage;
+            if (NS > 32) NS = 32;
+            if (NS < 2) NS = 2;
+        }
+        p.kv_splits = 1;
+        p.warps_per_cta = W;
+        p.stages = NS;
+        p.decode_ctas = d.ctas;
+        p.max_segments = d.max_seg;
+        p.decode_smem_bytes = c->head_dim == 64 ? lar::stream_smem_bytes(64, d.group, W, NS) : lar::stream_smem_bytes(128, d.group, W, NS);
+        return;
+    }
     const int tiles = (d.cap + lar::kGranule - 1) / lar::kGranule;  // tiles at the longest live length
     int X = c->kv_splits;
     if (X == 0) {
@@ -133,9 +177,9 @@ void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
     p.kv_splits = X;
     p.warps_per_cta = W;
     p.stages = NS;
-    p.decode_smem_bytes = c->dtype == LAR_BF16
-                              ? lar::decode_mma_smem_bytes(c->head_dim, W, NS, X, d.group)
-                              : lar::decode_smem_bytes(2 * lar::kGranule * d.row_bytes, W, NS, X, d.group, c->head_dim);
+    p.decode_ctas = d.units * X;
+    p.max_segments = 1;
+    p.decode_smem_bytes = lar::decode_smem_bytes(2 * lar::kGranule * d.row_bytes, W, NS, X, d.group, c->head_dim);
 }
 
 lar_status_t plan_query_impl(const lar_config_t* cfg, lar_plan_t* out, Derived* dout, Layout* lout) {
@@ -154,6 +198,7 @@ lar_status_t plan_query_impl(const lar_config_t* cfg, lar_plan_t* out, Derived* 
     p.line_end_smem_bytes =
         d.compressing ? lar::line_end_smem_bytes(d.row_bytes, cfg->head_dim, d.M, d.M - cfg->line_width + cfg->recent_lines * cfg->line_width, 8) : 0;
     p.slab_bytes = L.total;
+    p.scratch_bytes = (L.off_tickets + L.tickets_bytes) - L.off_partials;
     if (p.decode_smem_bytes > 227 * 1024 || p.line_end_smem_bytes > 227 * 1024) return LAR_ERR_INVALID_ARG;
     if (out) *out = p;
     if (dout) *dout = d;
@@ -254,19 +299,19 @@ lar_status_t make_tensor_maps(lar_cache* c) {
 }
 
 // ---- kernel tables ------------------------------------------------------------------------------
-using DecodeMmaFn = void (*)(const lar::DecodeArgs, const lar::TensorMaps, const int);
+using DecodeStreamFn = void (*)(const lar::StreamArgs, const lar::TensorMaps);
 template <int D>
-DecodeMmaFn decode_mma_for_group(int G) {
+DecodeStreamFn decode_stream_for_group(int G) {
     switch (G) {
-        case 1: return lar::decode_mma_kernel<D, 1>;
-        case 2: return lar::decode_mma_kernel<D, 2>;
-        case 4: return lar::decode_mma_kernel<D, 4>;
-        case 8: return lar::decode_mma_kernel<D, 8>;
+        case 1: return lar::decode_stream_kernel<D, 1>;
+        case 2: return lar::decode_stream_kernel<D, 2>;
+        case 4: return lar::decode_stream_kernel<D, 4>;
+        case 8: return lar::decode_stream_kernel<D, 8>;
     }
     return nullptr;
 }
-DecodeMmaFn decode_mma_fn(const lar_config_t& c, int G) {
-    return c.head_dim == 64 ? decode_mma_for_group<64>(G) : decode_mma_for_group<128>(G);
+DecodeStreamFn decode_stream_fn(const lar_config_t& c, int G) {
+    return c.head_dim == 64 ? decode_stream_for_group<64>(G) : decode_stream_for_group<128>(G);
 }
 using DecodeFn = void (*)(const lar::DecodeArgs);
 using LineEndFn = void (*)(const lar::LayerView, float);
@@ -322,45 +367,71 @@ lar_status_t launch_append(lar_cache* c, int layer, const void* k, const void* v
 
 lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k, const void* v, void* out, int fused,
                            cudaStream_t s) {
-    lar::DecodeArgs a;
-    a.lv = view_of(c, layer);
-    a.q = q;
-    a.k_new = k;
-    a.v_new = v;
-    a.out = out;
-    a.scale_log2 = c->scale * 1.4426950408889634f;
-    a.fused = fused;
     const bool pdl = (c->cfg.flags & LAR_FLAG_PDL) != 0;
-    a.prefetch = (pdl && c->last_layer != layer && c->last_layer >= 0) ? 1 : 0;
-    a.splits = c->plan.kv_splits;
-    a.stages = c->plan.stages;
+    const int prefetch = (pdl && c->last_layer != layer && c->last_layer >= 0) ? 1 : 0;
+    const float scale_log2 = c->scale * 1.4426950408889634f;
 
     cudaLaunchConfig_t lc;
     memset(&lc, 0, sizeof(lc));
-    lc.gridDim = dim3((unsigned)(c->d.units * c->plan.kv_splits), 1, 1);
-    lc.blockDim = dim3((unsigned)(32 * c->plan.warps_per_cta), 1, 1);
     lc.dynamicSmemBytes = (size_t)c->plan.decode_smem_bytes;
     lc.stream = s;
     cudaLaunchAttribute attrs[2];
     unsigned na = 0;
-    if (c->plan.kv_splits > 1) {
-        attrs[na].id = cudaLaunchAttributeClusterDimension;
-        attrs[na].val.clusterDim.x = (unsigned)c->plan.kv_splits;
-        attrs[na].val.clusterDim.y = 1;
-        attrs[na].val.clusterDim.z = 1;
-        ++na;
-    }
     if (pdl) {
         attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attrs[na].val.programmaticStreamSerializationAllowed = 1;
         ++na;
     }
-    lc.attrs = attrs;
-    lc.numAttrs = na;
     if (c->cfg.dtype == LAR_BF16) {
-        DecodeMmaFn fn = decode_mma_fn(c->cfg, c->d.group);
-        LAR_CUDA(cudaLaunchKernelEx(&lc, fn, a, c->tmaps, layer * c->rows_per_layer));
+        // bulk copies of q / k / v rows need 16-byte aligned sources
+        if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k) |
+             reinterpret_cast<uintptr_t>(v)) & 15u)
+            return LAR_ERR_INVALID_ARG;
+        lar::StreamArgs a;
+        a.lv = view_of(c, layer);
+        a.q = q;
+        a.k_new = k;
+        a.v_new = v;
+        a.out = out;
+        a.partials = reinterpret_cast<float*>(c->slab + c->L.off_partials);
+        a.tickets = reinterpret_cast<int*>(c->slab + c->L.off_tickets);
+        a.done = a.tickets + c->d.units;
+        a.scale_log2 = scale_log2;
+        a.fused = fused;
+        a.prefetch = prefetch;
+        a.n_units = c->d.units;
+        a.n_stages = c->plan.stages;
+        a.max_seg = c->d.max_seg;
+        a.pool_row_base = layer * c->rows_per_layer;
+        lc.gridDim = dim3((unsigned)c->d.ctas, 1, 1);
+        lc.blockDim = dim3((unsigned)(32 * (c->plan.warps_per_cta + 2)), 1, 1);
+        lc.attrs = attrs;
+        lc.numAttrs = na;
+        DecodeStreamFn fn = decode_stream_fn(c->cfg, c->d.group);
+        LAR_CUDA(cudaLaunchKernelEx(&lc, fn, a, c->tmaps));
     } else {
+        lar::DecodeArgs a;
+        a.lv = view_of(c, layer);
+        a.q = q;
+        a.k_new = k;
+        a.v_new = v;
+        a.out = out;
+        a.scale_log2 = scale_log2;
+        a.fused = fused;
+        a.prefetch = prefetch;
+        a.splits = c->plan.kv_splits;
+        a.stages = c->plan.stages;
+        lc.gridDim = dim3((unsigned)(c->d.units * c->plan.kv_splits), 1, 1);
+        lc.blockDim = dim3((unsigned)(32 * c->plan.warps_per_cta), 1, 1);
+        if (c->plan.kv_splits > 1) {
+            attrs[na].id = cudaLaunchAttributeClusterDimension;
+            attrs[na].val.clusterDim.x = (unsigned)c->plan.kv_splits;
+            attrs[na].val.clusterDim.y = 1;
+            attrs[na].val.clusterDim.z = 1;
+            ++na;
+        }
+        lc.attrs = attrs;
+        lc.numAttrs = na;
         DecodeFn fn = decode_fn(c->cfg, c->d.group);
         LAR_CUDA(cudaLaunchKernelEx(&lc, fn, a));
     }
@@ -463,8 +534,9 @@ lar_status_t lar_cache_create(const lar_config_t* cfg, void* dev_slab, size_t sl
     // rows of a page beyond the live length are read by short tiles with weight 0: they must be finite
     if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_kpool, 0, L.stride_pool * cfg->n_layers);
     if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_vpool, 0, L.stride_pool * cfg->n_layers);
+    if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_tickets, 0, L.tickets_bytes);
     if (ce == cudaSuccess)
-        ce = cudaFuncSetAttribute(cfg->dtype == LAR_BF16 ? (const void*)decode_mma_fn(*cfg, d.group) : (const void*)decode_fn(*cfg, d.group),
+        ce = cudaFuncSetAttribute(cfg->dtype == LAR_BF16 ? (const void*)decode_stream_fn(*cfg, d.group) : (const void*)decode_fn(*cfg, d.group),
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, plan.decode_smem_bytes);
     if (ce == cudaSuccess && d.compressing)
         ce = cudaFuncSetAttribute((const void*)line_end_fn(*cfg, d.group), cudaFuncAttributeMaxDynamicSharedMemorySize, plan.line_end_smem_bytes);
@@ -487,6 +559,7 @@ lar_status_t lar_cache_destroy(lar_cache_t* c) {
 lar_status_t lar_cache_reset(lar_cache_t* c, void* stream) {
     if (!c) return LAR_ERR_INVALID_ARG;
     LAR_CUDA(cudaMemsetAsync(c->slab + c->L.off_state, 0, c->L.stride_state * c->cfg.n_layers, (cudaStream_t)stream));
+    LAR_CUDA(cudaMemsetAsync(c->slab + c->L.off_tickets, 0, c->L.tickets_bytes, (cudaStream_t)stream));
     for (auto& s : c->sh) s = LayerShadow();
     c->last_layer = -1;
     return LAR_OK;

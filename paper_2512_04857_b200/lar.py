@@ -26,14 +26,15 @@ class lar_config_t(C.Structure):
                 ("n_lines", C.c_int32), ("anchor_len", C.c_int32), ("recent_lines", C.c_int32),
                 ("budget_lines", C.c_int32), ("softmax_scale", C.c_float), ("page_tokens", C.c_int32),
                 ("flags", C.c_uint32), ("kv_splits", C.c_int32), ("warps_per_cta", C.c_int32),
-                ("stages", C.c_int32), ("page_seed", C.c_uint32)]
+                ("stages", C.c_int32), ("page_seed", C.c_uint32), ("decode_ctas", C.c_int32)]
 
 
 class lar_plan_t(C.Structure):
     _fields_ = [("capacity", C.c_int32), ("pages_per_unit", C.c_int32), ("page_tokens", C.c_int32),
                 ("mid_len", C.c_int32), ("kv_splits", C.c_int32), ("warps_per_cta", C.c_int32),
                 ("stages", C.c_int32), ("decode_smem_bytes", C.c_int32), ("line_end_smem_bytes", C.c_int32),
-                ("compressing", C.c_int32), ("slab_bytes", C.c_uint64)]
+                ("compressing", C.c_int32), ("slab_bytes", C.c_uint64), ("decode_ctas", C.c_int32),
+                ("max_segments", C.c_int32), ("scratch_bytes", C.c_uint64)]
 
 
 class LarError(RuntimeError):
@@ -85,11 +86,12 @@ def lib():
 
 def make_config(*, n_layers, batch, n_q_heads, n_kv_heads, head_dim, dtype, cond_len, line_width, n_lines,
                 anchor_len, recent_lines, budget_lines, softmax_scale=0.0, page_tokens=0, flags=0,
-                kv_splits=0, warps_per_cta=0, stages=0, page_seed=0) -> lar_config_t:
+                kv_splits=0, warps_per_cta=0, stages=0, page_seed=0, decode_ctas=0) -> lar_config_t:
     dt = {"bf16": LAR_BF16, "fp32": LAR_FP32}.get(dtype, dtype)
     return lar_config_t(C.sizeof(lar_config_t), n_layers, batch, n_q_heads, n_kv_heads, head_dim, dt,
                         cond_len, line_width, n_lines, anchor_len, recent_lines, budget_lines,
-                        float(softmax_scale), page_tokens, flags, kv_splits, warps_per_cta, stages, page_seed)
+                        float(softmax_scale), page_tokens, flags, kv_splits, warps_per_cta, stages, page_seed,
+                        decode_ctas)
 
 
 def config_from_workload(w, **overrides) -> lar_config_t:

@@ -43,7 +43,10 @@ def test_plan_of_each_workload(name):
     assert p.capacity == w.cond_len + w.budget_tokens
     assert p.mid_len == w.mid_len and p.compressing == 1
     assert p.pages_per_unit * p.page_tokens >= p.capacity
-    assert p.kv_splits in (1, 2, 4, 8) and 1 <= p.warps_per_cta <= 8 and 1 <= p.stages <= 4
+    assert p.kv_splits in (1, 2, 4, 8) and 1 <= p.warps_per_cta <= 8 and 1 <= p.stages <= 32
+    assert p.decode_ctas >= 1 and 1 <= p.max_segments <= p.decode_ctas and p.scratch_bytes < p.slab_bytes
+    if w.dtype == "bf16":
+        assert 2 * (p.decode_smem_bytes + 1024) <= 228 * 1024      # two decode CTAs fit on one SM
     assert p.decode_smem_bytes <= 227 * 1024 and p.line_end_smem_bytes <= 227 * 1024
     kv = 2 * w.n_layers * w.n_units * p.pages_per_unit * p.page_tokens * w.head_dim * w.elt_bytes
     assert kv <= p.slab_bytes <= kv * 1.3 + (1 << 22)
@@ -70,7 +73,12 @@ def _cfg(**kw):
     dict(page_tokens=24),
     dict(kv_splits=3),
     dict(warps_per_cta=9),
-    dict(stages=5),
+    dict(stages=33),
+    dict(stages=1),                           # bf16 ring needs two stages
+    dict(dtype="fp32", stages=5),
+    dict(dtype="fp32", warps_per_cta=9),
+    dict(decode_ctas=-1),
+    dict(decode_ctas=2000),
     dict(n_layers=0),
     dict(cond_len=-1),
     dict(softmax_scale=-1.0),
@@ -109,5 +117,9 @@ def test_full_cache_budget_and_overrides():
     assert p.compressing == 0 and p.capacity == 4 + 64
     p = lar.lar_plan_query(_cfg(budget_lines=100))
     assert p.compressing == 0 and p.capacity == 4 + 64
-    p = lar.lar_plan_query(_cfg(kv_splits=4, warps_per_cta=8, stages=2, page_tokens=32))
+    p = lar.lar_plan_query(_cfg(dtype="fp32", kv_splits=4, warps_per_cta=8, stages=2, page_tokens=32))
     assert (p.kv_splits, p.warps_per_cta, p.stages, p.page_tokens) == (4, 8, 2, 32)
+    p = lar.lar_plan_query(_cfg(warps_per_cta=3, stages=9, decode_ctas=40, page_tokens=64))
+    assert (p.warps_per_cta, p.stages, p.decode_ctas, p.page_tokens) == (3, 9, 40, 64)
+    # 4 units of up to 3 tiles (36 slots) dealt to 40 CTAs: every tile may sit in a CTA of its own
+    assert p.max_segments == 3

@@ -44,6 +44,19 @@ def test_launch_shapes(splits, warps, stages):
     _check(rep, w)
 
 
+@pytest.mark.parametrize("ctas,warps,stages", [(1, 1, 2), (3, 2, 3), (7, 4, 5), (40, 3, 12), (148, 4, 0), (296, 1, 32),
+                                               (1024, 4, 2)])
+@pytest.mark.parametrize("fused", [True, False])
+def test_stream_launch_shapes_bf16(ctas, warps, stages, fused):
+    """bf16 streaming decode kernel: any grid size / ring depth / consumer count gives the same result,
+    including grids that cut every unit into many segments (scratch partials + ticket merge) and grids
+    with more CTAs than tiles."""
+    w = W.WORKLOADS["tiny_b"].scaled(dtype="bf16", n_q_heads=4, n_kv_heads=2, n_layers=2, cond_len=37)
+    rep = run_parity(w, fused=fused, cfg_overrides=dict(decode_ctas=ctas, warps_per_cta=warps, stages=stages,
+                                                        flags=lar.LAR_FLAG_PDL))
+    _check(rep, w, allow_near_ties=1)
+
+
 @pytest.mark.parametrize("page_tokens", [16, 32, 64])
 def test_shuffled_pages(page_tokens):
     w = W.WORKLOADS["tiny_b"]
