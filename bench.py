@@ -170,7 +170,7 @@ class Runner:
         if not args.no_pdl:
             flags |= lar.LAR_FLAG_PDL
         self.cfg = lar.config_from_workload(w, flags=flags, kv_splits=args.kv_splits, warps_per_cta=args.warps,
-                                            stages=args.stages, page_tokens=args.page_tokens)
+                                            stages=args.stages, page_tokens=args.page_tokens, decode_ctas=args.ctas)
         self.cache = lar.Cache(self.cfg, device=str(dev))
         L, S, Hq, Hkv, d, n, h = w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.line_width, w.n_lines
         dt = w.torch_dtype
@@ -305,7 +305,7 @@ def measure_e2e(w, dev, args, steps=1):
     from paper_2512_04857_b200 import lar, workloads as W
     flags = lar.LAR_FLAG_NO_HOST_CHECKS
     cfg = lar.config_from_workload(w, flags=flags, kv_splits=args.kv_splits, warps_per_cta=args.warps,
-                                   stages=args.stages, page_tokens=args.page_tokens)
+                                   stages=args.stages, page_tokens=args.page_tokens, decode_ctas=args.ctas)
     cache = lar.Cache(cfg, device=str(dev))
     L, S, Hq, Hkv, d, n, h = w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.line_width, w.n_lines
     dt = w.torch_dtype
@@ -388,7 +388,8 @@ def run_ours(args):
         res = {"ms_per_step": total_ms / steps, "decode_ms_per_step": decode_ms / steps, "clocks": clocks,
                "launches": r.launches_per_generation, "status_bits": bits,
                "plan": {"kv_splits": plan.kv_splits, "warps_per_cta": plan.warps_per_cta, "stages": plan.stages,
-                        "page_tokens": plan.page_tokens, "decode_smem_bytes": plan.decode_smem_bytes},
+                        "page_tokens": plan.page_tokens, "decode_smem_bytes": plan.decode_smem_bytes,
+                        "decode_ctas": plan.decode_ctas},
                "per_token_ms_first_half": halves[0], "per_token_ms_last_half": halves[1]}
         r.close()
         torch.cuda.empty_cache()
@@ -482,6 +483,7 @@ def main():
     ap.add_argument("--warps", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--page-tokens", type=int, default=0)
+    ap.add_argument("--ctas", type=int, default=0, help="CTAs of the persistent decode grid (0: one per SM)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling / small cases)")
     ap.add_argument("--eager", action="store_true", help="plain stream launches instead of CUDA graphs (profiling)")
     ap.add_argument("--no-pdl", action="store_true")

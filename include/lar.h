@@ -47,10 +47,14 @@ typedef enum {
 typedef enum { LAR_BF16 = 0, LAR_FP32 = 1 } lar_dtype_t;
 
 /* config.flags */
-#define LAR_FLAG_NO_HOST_CHECKS 0x1u /* skip the host-side call-order checks (needed when calls are
-                                        captured once into a CUDA graph and replayed: the host-side
-                                        counters then no longer follow the device). Device-side
-                                        checks stay active. */
+#define LAR_FLAG_NO_HOST_CHECKS 0x1u /* skip the host-side call-order checks.  Needed when calls are captured
+                                        into CUDA graphs: the host-side counters advance at capture, not at
+                                        replay.  The live length of a step is a closed form of the step index
+                                        and is passed to the decode kernel by the host, so a graph holds the
+                                        lengths of the steps it was captured at: capture the calls of a
+                                        generation in order and replay the graphs in that same order (the
+                                        kernels check the length against device memory and record bit 16
+                                        otherwise).  Device-side checks stay active. */
 #define LAR_FLAG_PDL 0x2u            /* launch decode kernels with programmatic dependent launch and
                                         let them prefetch cached K/V before the preceding kernel on the
                                         stream has finished.  Contract: the kernel enqueued on `stream`
@@ -59,6 +63,8 @@ typedef enum { LAR_BF16 = 0, LAR_FP32 = 1 } lar_dtype_t;
                                         caller kernel using PDL waits on its own dependency before it
                                         triggers its dependents. */
 #define LAR_FLAG_SHUFFLE_PAGES 0x4u  /* test hook: assign physical pages in a pseudo-random order */
+#define LAR_FLAG_TILE_RANGES 0x8u    /* bf16 decode: always deal 16-row tiles (not whole units) to the CTAs, even
+                                        where whole units would balance well enough */
 
 typedef struct lar_config {
     uint32_t struct_size;  /* = sizeof(lar_config_t) */
@@ -80,7 +86,8 @@ typedef struct lar_config {
     int32_t kv_splits;     /* fp32 only: CTAs (one thread-block cluster) per unit in decode: 0 auto, else 1,2,4,8 */
     int32_t warps_per_cta; /* decode warps: bf16 consumer warps per CTA, 0 auto, else 1..4;
                               fp32 warps per CTA, 0 auto, else 1..8 */
-    int32_t stages;        /* 16-row K/V stages: bf16 depth of the CTA's ring, 0 auto, else 2..32;
+    int32_t stages;        /* 16-row K/V stages: bf16 depth of the CTA's ring, 0 auto, else 2..32 (rounded
+                              down to a multiple of the consumer warps, at least one per warp);
                               fp32 stages in flight per warp, 0 auto, else 1..4 */
     uint32_t page_seed;    /* seed of LAR_FLAG_SHUFFLE_PAGES */
     int32_t decode_ctas;   /* bf16 only: CTAs of the persistent decode grid: 0 selects 148 (one per SM), else 1..1024 */
@@ -169,7 +176,8 @@ lar_status_t lar_cache_get_state(lar_cache_t* c, int layer, int32_t* lens, int32
 
 /* Synchronises `stream` and returns LAR_ERR_DEVICE_CHECK if any kernel recorded a failed check since
  * the last poll (bits in *bits_out, may be NULL: 1 capacity, 2 line-end off boundary, 4 wait limit,
- * 8 decode on an empty cache); clears the word. */
+ * 8 decode on an empty cache, 16 the length the host passed to a decode kernel differs from
+ * the device's, e.g. a captured graph replayed out of order); clears the word. */
 lar_status_t lar_cache_poll_device_status(lar_cache_t* c, uint32_t* bits_out, void* stream);
 
 /* Enable (1) / disable (0) the host-side call-order checks at run time (see LAR_FLAG_NO_HOST_CHECKS). */

@@ -2,12 +2,16 @@
 // fused with the append of the step's token (Eq. 4) and the guide-queue push (Eq. 8).
 //
 // Work decomposition.  The live rows of every unit = (sequence, KV head) are cut into 16-row tiles;
-// all tiles of the layer form one list (unit-major) that is dealt out in equal contiguous ranges
-// to the CTAs of the grid (one CTA per SM), so every SM streams the same number of bytes whatever
-// the number of units.  The part of a unit that falls into one CTA is a *segment*.  A unit that lies
-// inside one CTA is finished there; a unit cut by a range boundary leaves one partial (m, l, o) per
-// segment in a global scratch area and the CTA that delivers the last partial (an atomic ticket, no
-// waiting) merges them.
+// all tiles of the layer form one list (unit-major) that is dealt out in contiguous ranges to the CTAs
+// of the grid (one CTA per SM).  Where whole units can be dealt out evenly enough the ranges end on unit
+// boundaries; otherwise they are equal in tiles, so that every SM streams the same number of bytes
+// whatever the number of units.  The part of a unit that falls into one CTA is a *segment*.  A unit
+// that lies inside one CTA is finished there; a unit cut by a range boundary leaves one partial
+// (m, l, o) per segment in a global scratch area and the CTA that delivers the last partial (an atomic
+// ticket, no waiting) merges them.
+// The live length is the same for every unit (sequences decode in lock-step) and is a closed form of
+// the step index; the host passes it, so that all CTAs agree on the tile list, and the CTA that closes a
+// unit checks it against the unit's length in device memory before advancing that.
 //
 // Inside a CTA three roles run concurrently, coupled only by mbarriers (every wait is bounded):
 //   warp 0           producer: walks the CTA's tile range and keeps a ring of NS stages filled with
@@ -32,8 +36,9 @@
 namespace lar {
 
 struct TensorMaps {
-    CUtensorMap k[4];  // box heights 4, 8, 12, 16 rows over the K pools of all layers
-    CUtensorMap v[4];
+    // 3-D maps over {head_dim, pool rows of all layers, {K pool, V pool}}: one copy brings the K rows and
+    // the V rows of a tile; box = 64 elements x 4 (i + 1) rows x 2
+    CUtensorMap kv[4];
 };
 
 struct StreamArgs {
@@ -44,18 +49,19 @@ struct StreamArgs {
     void* out;          // [units * G][d]
     float* partials;    // scratch [units][max_seg][G][d + 2]
     int* tickets;       // scratch [units], zero between launches
-    int* done;          // scratch, one counter, zero between launches
     float scale_log2;   // softmax scale * log2(e)
+    int len, n_tok;     // live rows per unit / visual tokens appended so far, before this step's append
+    int unit_ranges;    // 1: CTA ranges end on unit boundaries
     int fused;          // 1: the step's token comes from k_new / v_new and is appended by this kernel
     int prefetch;       // 1: cached K/V may be fetched before the preceding kernel has finished
     int n_units, n_stages, max_seg;
     int pool_row_base;  // first pool row of this layer in the tensor maps
 };
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
@@ -85,18 +91,19 @@ __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_
 template <int D>
 struct MmaTraits {
     static constexpr int ROW_BYTES = D * 2;
-    static constexpr int HALVES = D / 64;             // 128-byte column blocks per row
-    static constexpr int SUB_BYTES = kGranule * 128;  // one [16][64] swizzled block
-    static constexpr int TILE_BYTES = HALVES * SUB_BYTES;
-    static constexpr int STAGE_BYTES = 2 * TILE_BYTES;  // K tile + V tile
+    static constexpr int HALVES = D / 64;                  // 128-byte column blocks per row
+    static constexpr int HALF_BYTES = 2 * kGranule * 128;  // one swizzled block: [K rows | V rows][64 elements]
+    static constexpr int STAGE_BYTES = HALVES * HALF_BYTES;
     static constexpr int KSTEPS = D / 16;
     static constexpr int NTILES = D / 8;
 };
 
-// byte offset of 16-byte chunk `c` of row `r` inside a tile stored as HALVES swizzled [16][128 B] blocks
+// A stage holds HALVES blocks of 128-byte lines; a block is what one copy of box height b delivers: lines
+// 0 .. b-1 are the K rows, lines b .. 2b-1 the V rows (128-byte swizzle on the line index).
+// Byte offset of 16-byte chunk `c` of line `r` of a stage:
 template <int D>
 __device__ __forceinline__ uint32_t tile_off(int r, int c) {
-    return (uint32_t)((c >> 3) * MmaTraits<D>::SUB_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+    return (uint32_t)((c >> 3) * MmaTraits<D>::HALF_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
 // ---- shared-memory plan of decode_stream_kernel (host and device agree through these) -------------
@@ -138,7 +145,7 @@ __device__ __forceinline__ float exp2_or_zero(float m_part, float m_all) {
     return m_part == -INFINITY ? 0.f : exp2f(m_part - m_all);
 }
 
-// CTA that owns tile t of a list of `total` tiles dealt to P <= total CTAs as ranges [p total / P, (p + 1) total / P)
+// CTA that owns item t of a list of `total` items dealt to P <= total CTAs as ranges [p total / P, (p + 1) total / P)
 __device__ __forceinline__ int range_owner(long long t, long long total, int P) {
     return (int)(((t + 1) * P - 1) / total);
 }
@@ -192,13 +199,25 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
 
     if (!a.prefetch) grid_dep_wait();
 
-    // ---- the layer's tile list and this CTA's range of it (units decode in lock-step: one length)
-    const int len = __ldcg(&lv.state[0].len);
-    const int n_tok = __ldcg(&lv.state[0].n_tok);
+    // ---- the layer's tile list and this CTA's range of it
+    const int len = a.len, n_tok = a.n_tok;
     const int T = len > 0 ? (len + kGranule - 1) / kGranule : 1;  // an empty cache is one tile of 0 rows
     const long long total = (long long)a.n_units * T;
-    const int Pe = total < P ? (int)total : P;  // CTAs that get tiles: every range is non-empty
-    const long long t_begin = p < Pe ? (long long)p * total / Pe : 0, t_end = p < Pe ? (long long)(p + 1) * total / Pe : 0;
+    long long t_begin = 0, t_end = 0;
+    int Pe;  // CTAs that get work: every range is non-empty
+    if (a.unit_ranges) {
+        Pe = a.n_units < P ? a.n_units : P;
+        if (p < Pe) {
+            t_begin = ((long long)p * a.n_units / Pe) * T;
+            t_end = ((long long)(p + 1) * a.n_units / Pe) * T;
+        }
+    } else {
+        Pe = total < P ? (int)total : P;
+        if (p < Pe) {
+            t_begin = (long long)p * total / Pe;
+            t_end = (long long)(p + 1) * total / Pe;
+        }
+    }
     const int n_tiles = (int)(t_end - t_begin);
     const int u0 = (int)(t_begin / T);
     const int n_segs = n_tiles > 0 ? (int)((t_end - 1) / T) - u0 + 1 : 0;
@@ -239,37 +258,48 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
             return true;
         };
 
-        int y_n = 0, rows_n = 0, tile_n = 0;
-        if (lane < n_tiles) describe(lane, y_n, rows_n, tile_n);
-        for (int j0 = 0; j0 < n_tiles && ok; j0 += 32) {
-            const int y = y_n, rows = rows_n, tile = tile_n;
-            if (j0 + 32 + lane < n_tiles) describe(j0 + 32 + lane, y_n, rows_n, tile_n);  // next batch: hides the table reads
+        // Lane 0 issues; all lanes look the page ids of a batch of 32 tiles up together, one batch ahead.
+        // Stage and phase advance incrementally (no division in the per-tile path).  A fresh mbarrier lets a
+        // wait on parity 1 pass, so the first trip round the ring does not wait for the consumers.
+        int y_n = 0, rt_n = 0;  // rt = rows | tile << 8
+        {
+            int r = 0, t = 0;
+            if (lane < n_tiles) describe(lane, y_n, r, t);
+            rt_n = r | (t << 8);
+        }
+        int stage = 0;
+        uint32_t empty_parity = 1;
+        for (int j0 = 0; j0 < n_tiles; j0 += 32) {
+            const int y = y_n, rt = rt_n;
+            if (j0 + 32 + lane < n_tiles) {  // next batch: hides the table reads
+                int r = 0, t = 0;
+                describe(j0 + 32 + lane, y_n, r, t);
+                rt_n = r | (t << 8);
+            }
             const int cnt = n_tiles - j0 < 32 ? n_tiles - j0 : 32;
             for (int i = 0; i < cnt; ++i) {
                 const int j = j0 + i;
-                const int yi = __shfl_sync(0xffffffffu, y, i), ri = __shfl_sync(0xffffffffu, rows, i);
-                const int ti = __shfl_sync(0xffffffffu, tile, i);
-                if (lane == 0) {
-                    if (dep_waited && (j == 0 || ti == 0)) ok = issue_inputs(q_next++);
-                    const int s = j % NS;
-                    if (ok && j >= NS) ok = wait_or_abort(bar_empty + s * 8, (uint32_t)((j / NS - 1) & 1), abort_flag);
+                const int yi = __shfl_sync(0xffffffffu, y, i), rti = __shfl_sync(0xffffffffu, rt, i);
+                if (lane == 0 && ok) {
+                    const int ri = rti & 0xff;
+                    if (dep_waited && (j == 0 || (rti >> 8) == 0)) ok = issue_inputs(q_next++);
+                    if (ok) ok = wait_or_abort(bar_empty + stage * 8, empty_parity, abort_flag);
                     if (ok) {
-                        const uint32_t bar = bar_full + s * 8, dst = ring + (uint32_t)s * TR::STAGE_BYTES;
+                        const uint32_t bar = bar_full + stage * 8, dst = ring + (uint32_t)stage * TR::STAGE_BYTES;
                         if (ri > 0) {
                             const int hsel = (ri + 3) / 4 - 1;  // box of 4 * (hsel + 1) rows
                             mbar_expect_tx(bar, (uint32_t)(2 * 4 * (hsel + 1) * TR::ROW_BYTES));
 #pragma unroll
-                            for (int h = 0; h < TR::HALVES; ++h) {
-                                tma_load_2d(dst + h * TR::SUB_BYTES, &tm.k[hsel], h * 64, yi, bar);
-                                tma_load_2d(dst + TR::TILE_BYTES + h * TR::SUB_BYTES, &tm.v[hsel], h * 64, yi, bar);
-                            }
+                            for (int h = 0; h < TR::HALVES; ++h) tma_load_3d(dst + h * TR::HALF_BYTES, &tm.kv[hsel], h * 64, yi, 0, bar);
                         } else {
                             mbar_arrive(bar);  // nothing to fetch: release the consumer
                         }
                     }
+                    if (++stage == NS) {
+                        stage = 0;
+                        empty_parity ^= 1u;
+                    }
                 }
-                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                if (!ok) break;
                 if (!dep_waited && j == fill_end - 1) {
                     // the ring is full of this layer's cache; everything else depends on the preceding kernel
                     grid_dep_wait();
@@ -279,8 +309,6 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
                         const int seg_now = (int)((t_begin + j) / T) - u0;
                         while (ok && q_next <= seg_now) ok = issue_inputs(q_next++);
                     }
-                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                    if (!ok) break;
                 }
             }
         }
@@ -296,10 +324,13 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
         const int cw = warp - 1;
         const int quad = lane & 3, qrow = lane >> 2;  // fragment coordinates
         bool ok = true;
+        // This consumer takes tiles cw, cw + W, ... of the CTA's range.  NS is a multiple of W, so a stage is
+        // always read by the same consumer, which has seen every earlier phase of its barrier.
+        int j = cw, stage = cw;
+        uint32_t full_parity = 0;
         for (int seg = 0; seg < n_segs && ok; ++seg) {
             const int unit = u0 + seg;
             const long long ub = (long long)unit * T;
-            const int jb = (int)((ub > t_begin ? ub : t_begin) - t_begin);
             const int je = (int)((ub + T < t_end ? ub + T : t_end) - t_begin);
 
             // ---- Q fragments (A operand): row qrow = head, 16 columns per k-step; heads >= G are zero rows
@@ -327,34 +358,40 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
 #pragma unroll
             for (int t = 0; t < TR::NTILES; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
 
-            for (int j = jb + ((cw - jb % W) + W) % W; j < je; j += W) {
-                const int s = j % NS;
-                ok = wait_or_abort(bar_full + s * 8, (uint32_t)((j / NS) & 1), abort_flag);
+            for (; j < je; j += W) {
+                const int s = stage;
+                ok = wait_or_abort(bar_full + s * 8, full_parity, abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+                stage += W;
+                if (stage >= NS) {
+                    stage -= NS;
+                    full_parity ^= 1u;
+                }
                 const int tile = (int)(t_begin + j - ub);
                 const int rows = len - tile * kGranule < kGranule ? len - tile * kGranule : kGranule;
-                const uint32_t Ks = ring + (uint32_t)s * TR::STAGE_BYTES;
-                const uint32_t Vs = Ks + TR::TILE_BYTES;
+                const uint32_t St = ring + (uint32_t)s * TR::STAGE_BYTES;
                 if (rows > 0) {
-                    // S[head][key] for the 16 keys of the tile: two n-tiles of 8 keys
-                    float sc[2][4];
+                    const int box_rows = (rows + 3) & ~3;  // K rows are lines 0.., V rows lines box_rows.. of a block
+                    // S[head][key] for the 16 keys of the tile: two n-tiles of 8 keys, two accumulators each
+                    float sc[2][2][4];
 #pragma unroll
                     for (int jn = 0; jn < 2; ++jn) {
-                        sc[jn][0] = sc[jn][1] = sc[jn][2] = sc[jn][3] = 0.f;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) sc[jn][0][e] = sc[jn][1][e] = 0.f;
 #pragma unroll
                         for (int i = 0; i < TR::KSTEPS / 2; ++i) {
                             uint32_t b[4];
-                            ldmatrix_x4(Ks + tile_off<D>(8 * jn + (lane & 7), 4 * i + (lane >> 3)), b);
-                            mma_bf16(sc[jn], qa0[2 * i], 0u, qa2[2 * i], 0u, b[0], b[1]);
-                            mma_bf16(sc[jn], qa0[2 * i + 1], 0u, qa2[2 * i + 1], 0u, b[2], b[3]);
+                            ldmatrix_x4(St + tile_off<D>(8 * jn + (lane & 7), 4 * i + (lane >> 3)), b);
+                            mma_bf16(sc[jn][0], qa0[2 * i], 0u, qa2[2 * i], 0u, b[0], b[1]);
+                            mma_bf16(sc[jn][1], qa0[2 * i + 1], 0u, qa2[2 * i + 1], 0u, b[2], b[3]);
                         }
                     }
                     // online softmax over the keys this thread holds: 2*quad, 2*quad+1 (+8)
                     float sv[4];
 #pragma unroll
                     for (int jn = 0; jn < 2; ++jn) {
-                        sv[2 * jn + 0] = (8 * jn + 2 * quad + 0 < rows) ? sc[jn][0] * a.scale_log2 : -INFINITY;
-                        sv[2 * jn + 1] = (8 * jn + 2 * quad + 1 < rows) ? sc[jn][1] * a.scale_log2 : -INFINITY;
+                        sv[2 * jn + 0] = (8 * jn + 2 * quad + 0 < rows) ? (sc[jn][0][0] + sc[jn][1][0]) * a.scale_log2 : -INFINITY;
+                        sv[2 * jn + 1] = (8 * jn + 2 * quad + 1 < rows) ? (sc[jn][0][1] + sc[jn][1][1]) * a.scale_log2 : -INFINITY;
                     }
                     float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
                     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
@@ -371,13 +408,13 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
                         for (int t = 0; t < TR::NTILES; ++t) { o[t][0] *= corr; o[t][1] *= corr; }
                     }
                     const uint32_t pa0 = pack_bf16(pr[0], pr[1]), pa2 = pack_bf16(pr[2], pr[3]);
-                    // a short box leaves rows of the V tile unwritten: their weight is 0, but 0 * (stale NaN) is not
-                    const int box_rows = (rows + 3) & ~3;
+                    // a short box leaves the lines behind its V rows unwritten: their weight is 0, but
+                    // 0 * (stale NaN) is not
                     if (box_rows < kGranule) {
-                        const int n16 = (kGranule - box_rows) * 8;  // 16-byte chunks per 128-byte-wide block
+                        const int n16 = (kGranule - box_rows) * 8;  // 16-byte chunks per block
                         for (int i = lane; i < n16 * TR::HALVES; i += 32) {
                             const int h = i / n16, c = i - h * n16;
-                            asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(Vs + h * TR::SUB_BYTES + box_rows * 128 + c * 16), "r"(0u) : "memory");
+                            asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(St + h * TR::HALF_BYTES + 2 * box_rows * 128 + c * 16), "r"(0u) : "memory");
                         }
                         __syncwarp();
                     }
@@ -385,7 +422,7 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
 #pragma unroll
                     for (int t = 0; t < TR::NTILES / 2; ++t) {
                         uint32_t b[4];
-                        ldmatrix_x4_trans(Vs + tile_off<D>((lane & 7) + 8 * ((lane >> 3) & 1), 2 * t + (lane >> 4)), b);
+                        ldmatrix_x4_trans(St + tile_off<D>(box_rows + (lane & 7) + 8 * ((lane >> 3) & 1), 2 * t + (lane >> 4)), b);
                         mma_bf16(o[2 * t], pa0, 0u, pa2, 0u, b[0], b[1]);
                         mma_bf16(o[2 * t + 1], pa0, 0u, pa2, 0u, b[2], b[3]);
                     }
@@ -424,11 +461,26 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
         grid_dep_launch();
         bool ok = true;
         T16* outp = reinterpret_cast<T16*>(a.out);
-        for (int seg = 0; seg < n_segs && ok; ++seg) {
+        // What closing a unit needs from global memory (the page that takes the new row, the unit's length
+        // in device memory) is requested one segment ahead, so that its latency never stalls this warp.
+        const int new_page_idx = len / lv.page_tokens;
+        auto closing_loads = [&](int sg, int& page, int& dev_len) {
+            const int un = u0 + sg;
+            page = 0;
+            dev_len = len;
+            if (sg < n_segs && (long long)(un + 1) * T <= t_end) {
+                if (a.fused && len < lv.cap) page = __ldg(&lv.page_table[un * lv.pages_per_unit + new_page_idx]);
+                dev_len = __ldcg(&lv.state[un].len);
+            }
+        };
+        int page_cur, dev_len_cur, page_nxt = 0, dev_len_nxt = 0;
+        closing_loads(0, page_cur, dev_len_cur);
+        for (int seg = 0; seg < n_segs && ok; ++seg, page_cur = page_nxt, dev_len_cur = dev_len_nxt) {
             const int unit = u0 + seg;
             const long long ub = (long long)unit * T;
             const bool opens = ub >= t_begin, closes = ub + T <= t_end;
             const int qs = seg % NQ, buf = seg & 1;
+            closing_loads(seg + 1, page_nxt, dev_len_nxt);
             ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             const unsigned char* Qs = qring_ptr + qs * QENT;
@@ -461,7 +513,7 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
                         s_new[g] = sv * a.scale_log2;
                     }
                     if (len < lv.cap) {
-                        const size_t off = row_offset(lv, unit, len, TR::ROW_BYTES);
+                        const size_t off = ((size_t)page_cur * lv.page_tokens + len % lv.page_tokens) * TR::ROW_BYTES;
                         const uint32_t* K32 = reinterpret_cast<const uint32_t*>(K16);
                         const uint32_t* V32 = reinterpret_cast<const uint32_t*>(V16);
                         for (int i = lane; i < D / 2; i += 32) {
@@ -474,6 +526,15 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
                     }
                 } else if (!a.fused && len == 0 && lane == 0) {
                     atomicOr(lv.status, kStEmpty);
+                }
+                if (lane == 0) {
+                    if (dev_len_cur != len) atomicOr(lv.status, kStLength);
+                    if (a.fused) {
+                        UnitState ns;
+                        ns.len = len < lv.cap ? len + 1 : len;
+                        ns.n_tok = n_tok + 1;
+                        lv.state[unit] = ns;
+                    }
                 }
                 // Eq. 8: the queries join the guide queue of the line being generated
                 const int tok = a.fused ? n_tok : n_tok - 1;  // 0-based visual index of this step's token
@@ -577,24 +638,6 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
             }
         }
         if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
-
-        // ---- the CTA that finishes last advances the lengths (nobody reads them any more in this launch)
-        __syncwarp();
-        int last = 0;
-        if (lane == 0) {
-            __threadfence();
-            last = atomicAdd(a.done, 1) == P - 1 ? 1 : 0;
-        }
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (last) {
-            if (a.fused) {
-                UnitState ns;
-                ns.len = len < lv.cap ? len + 1 : len;
-                ns.n_tok = n_tok + 1;
-                for (int u = lane; u < a.n_units; u += 32) lv.state[u] = ns;
-            }
-            if (lane == 0) *a.done = 0;
-        }
     }
 
     // ---- a role gave up: let the copies still in flight land before the shared memory is released

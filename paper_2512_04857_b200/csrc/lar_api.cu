@@ -49,6 +49,7 @@ struct Layout {
 struct Derived {
     int units, group, elt, row_bytes, cap, ppu, P, cap_pad, M, mid_pad, compressing, B, N;
     int ctas, max_seg;  // bf16 decode: CTAs of the persistent grid, most segments one unit is cut into
+    int unit_ranges;    // bf16 decode: 1 if the CTAs' ranges end on unit boundaries
 };
 
 constexpr int kDefaultDecodeCtas = 148;  // one per SM of a B200
@@ -93,6 +94,12 @@ bool derive(const lar_config_t* c, Derived& d) {
     d.mid_pad = (int)align_up((size_t)(d.M > 0 ? d.M : 1), 4);
     // A unit of T tiles is cut into at most ceil(T / floor(U T / P)) + 1 segments (never more than T or P).
     d.ctas = c->decode_ctas ? c->decode_ctas : kDefaultDecodeCtas;
+    // Whole units per CTA when that leaves at most ~6 % of imbalance: no unit is cut, nothing to merge.
+    {
+        const long long per = ((long long)d.units + d.ctas - 1) / d.ctas;
+        d.unit_ranges = (d.units >= d.ctas && per * d.ctas * 100 <= (long long)d.units * 106) ? 1 : 0;
+        if (c->flags & LAR_FLAG_TILE_RANGES) d.unit_ranges = 0;
+    }
     d.max_seg = 1;
     const int t_max = (d.cap + lar::kGranule - 1) / lar::kGranule;
     for (int T = 1; T <= t_max; ++T) {
@@ -130,7 +137,7 @@ void make_layout(const lar_config_t* c, const Derived& d, Layout& L) {
     L.off_kpool = take(L.stride_pool * Lyr);
     L.off_vpool = take(L.stride_pool * Lyr);
     L.off_partials = take(c->dtype == LAR_BF16 ? U * d.max_seg * d.group * (c->head_dim + 2) * sizeof(float) : 0);
-    L.tickets_bytes = (U + 1) * sizeof(int);  // one ticket per unit + the CTA counter
+    L.tickets_bytes = U * sizeof(int);  // one ticket per unit
     L.off_tickets = take(L.tickets_bytes);
     L.total = off;
 }
@@ -151,8 +158,11 @@ void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
             const int fixed = c->head_dim == 64 ? lar::stream_fixed_smem_bytes(64, d.group, W) : lar::stream_fixed_smem_bytes(128, d.group, W);
             NS = (budget - fixed) / stage;
             if (NS > 32) NS = 32;
-            if (NS < 2) NS = 2;
         }
+        // a stage must always be read by the same consumer warp: ring depth = a multiple of W
+        NS = NS / W * W;
+        if (NS < W) NS = W;
+        if (NS < 2) NS = 2;
         p.kv_splits = 1;
         p.warps_per_cta = W;
         p.stages = NS;
@@ -278,21 +288,18 @@ lar_status_t make_tensor_maps(lar_cache* c) {
     }
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fp);
     c->rows_per_layer = (int)(c->L.stride_pool / (size_t)c->d.row_bytes);
-    const cuuint64_t gdim[2] = {(cuuint64_t)c->cfg.head_dim, (cuuint64_t)c->rows_per_layer * (cuuint64_t)c->cfg.n_layers};
-    const cuuint64_t gstride[1] = {(cuuint64_t)c->d.row_bytes};
-    const cuuint32_t estr[2] = {1, 1};
+    // {head_dim, pool rows of all layers, {K pool, V pool}}
+    const cuuint64_t gdim[3] = {(cuuint64_t)c->cfg.head_dim, (cuuint64_t)c->rows_per_layer * (cuuint64_t)c->cfg.n_layers, 2};
+    const cuuint64_t gstride[2] = {(cuuint64_t)c->d.row_bytes, (cuuint64_t)(c->L.off_vpool - c->L.off_kpool)};
+    const cuuint32_t estr[3] = {1, 1, 1};
     for (int h = 0; h < 4; ++h) {
-        const cuuint32_t box[2] = {64, (cuuint32_t)(4 * (h + 1))};
-        for (int kv = 0; kv < 2; ++kv) {
-            CUtensorMap* m = kv == 0 ? &c->tmaps.k[h] : &c->tmaps.v[h];
-            void* base = c->slab + (kv == 0 ? c->L.off_kpool : c->L.off_vpool);
-            CUresult r = encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box, estr,
-                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-            if (r != CUDA_SUCCESS) {
-                g_last_cuda_error = (int)cudaErrorInvalidValue;
-                return LAR_ERR_CUDA;
-            }
+        const cuuint32_t box[3] = {64, (cuuint32_t)(4 * (h + 1)), 2};
+        CUresult r = encode(&c->tmaps.kv[h], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, c->slab + c->L.off_kpool, gdim, gstride, box,
+                            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            g_last_cuda_error = (int)cudaErrorInvalidValue;
+            return LAR_ERR_CUDA;
         }
     }
     return LAR_OK;
@@ -395,7 +402,15 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
         a.out = out;
         a.partials = reinterpret_cast<float*>(c->slab + c->L.off_partials);
         a.tickets = reinterpret_cast<int*>(c->slab + c->L.off_tickets);
-        a.done = a.tickets + c->d.units;
+        {
+            // live rows before this step's append, from the host-side counters (they follow the device's by
+            // construction: every call that changes the length updates both)
+            const LayerShadow& sh = c->sh[layer];
+            const int live = (sh.prefilled ? c->cfg.cond_len : 0) + sh.v;
+            a.len = live < c->d.cap ? live : c->d.cap;
+            a.n_tok = sh.n_tok;
+        }
+        a.unit_ranges = c->d.unit_ranges;
         a.scale_log2 = scale_log2;
         a.fused = fused;
         a.prefetch = prefetch;

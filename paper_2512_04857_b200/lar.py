@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "liblar.so")
 LAR_OK, LAR_ERR_INVALID_ARG, LAR_ERR_BAD_STATE, LAR_ERR_CAPACITY, LAR_ERR_CUDA, LAR_ERR_NOMEM, \
     LAR_ERR_DEVICE_CHECK = range(7)
 LAR_BF16, LAR_FP32 = 0, 1
-LAR_FLAG_NO_HOST_CHECKS, LAR_FLAG_PDL, LAR_FLAG_SHUFFLE_PAGES = 0x1, 0x2, 0x4
+LAR_FLAG_NO_HOST_CHECKS, LAR_FLAG_PDL, LAR_FLAG_SHUFFLE_PAGES, LAR_FLAG_TILE_RANGES = 0x1, 0x2, 0x4, 0x8
 
 
 class lar_config_t(C.Structure):
