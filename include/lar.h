@@ -84,7 +84,7 @@ typedef struct lar_config {
     int32_t page_tokens;   /* tokens per physical page: 16, 32 or 64; 0 selects 16 */
     uint32_t flags;        /* LAR_FLAG_* */
     int32_t kv_splits;     /* fp32 only: CTAs (one thread-block cluster) per unit in decode: 0 auto, else 1,2,4,8 */
-    int32_t warps_per_cta; /* decode warps: bf16 consumer warps per CTA, 0 auto, else 1..4;
+    int32_t warps_per_cta; /* decode warps: bf16 consumer warps per CTA, 0 auto, else 1..6;
                               fp32 warps per CTA, 0 auto, else 1..8 */
     int32_t stages;        /* 16-row K/V stages: bf16 depth of the CTA's ring, 0 auto, else 2..32 (rounded
                               down to a multiple of the consumer warps, at least one per warp);

@@ -20,7 +20,9 @@
 //   warps 1 .. W     consumers: tile j of the range goes to consumer j % W:
 //                        S = Q K^T     mma.sync m16n8k16 (bf16 in, fp32 out), rows = the G heads
 //                        online softmax in fp32 (base-2, scale folded into the logits)
-//                        O += P V      same instruction, V fragments via ldmatrix.trans
+//                        O^T += V^T P^T  same instruction with the d rows as M: the logits' accumulator
+//                                      layout is the B-operand layout of P^T, V^T fragments come from
+//                                      ldmatrix.trans, and no accumulator row is wasted on padding
 //                    and at the end of a segment each consumer leaves its partial in shared memory.
 //   warp W + 1       epilogue: merges the W partials of a segment with the step's own token,
 //                    writes the output row (or the scratch partial + ticket), stores the new K/V
@@ -136,6 +138,23 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
     }
     return true;
 }
+// ---- optional in-kernel timeline (builds with -DLAR_TRACE only): per CTA 32 words; time stamps are
+// %globaltimer ns, waits are accumulated SM clocks of the recording warp's lane 0
+#ifdef LAR_TRACE
+__device__ unsigned long long lar_trace_buf[1024 * 32];
+__device__ __forceinline__ unsigned long long trace_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define LAR_STAMP(slot) do { if ((threadIdx.x & 31) == 0) lar_trace_buf[blockIdx.x * 32 + (slot)] = trace_now(); } while (0)
+#define LAR_WAIT(slot, rec, call) [&]() { const long long t0__ = clock64(); const bool r__ = (call); \
+    if ((rec) && (threadIdx.x & 31) == 0) atomicAdd(&lar_trace_buf[blockIdx.x * 32 + (slot)], (unsigned long long)(clock64() - t0__)); return r__; }()
+#else
+#define LAR_STAMP(slot) do { } while (0)
+#define LAR_WAIT(slot, rec, call) (call)
+#endif
+
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -151,7 +170,7 @@ __device__ __forceinline__ int range_owner(long long t, long long total, int P) 
 }
 
 template <int D, int G>
-__global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs a, const __grid_constant__ TensorMaps tm) {
+__global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs a, const __grid_constant__ TensorMaps tm) {
     using TR = MmaTraits<D>;
     using T16 = __nv_bfloat16;
     constexpr int NQ = stream_q_slots(G);
@@ -197,6 +216,7 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
     }
     __syncthreads();
 
+    if (threadIdx.x == 0) LAR_STAMP(0);
     if (!a.prefetch) grid_dep_wait();
 
     // ---- the layer's tile list and this CTA's range of it
@@ -244,7 +264,7 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
         };
         auto issue_inputs = [&](int seg) -> bool {  // lane 0: q (and the step's k, v) of segment `seg`
             const int slot = seg % NQ;
-            if (seg >= NQ && !wait_or_abort(bar_qempty + slot * 8, (uint32_t)((seg / NQ - 1) & 1), abort_flag)) return false;
+            if (seg >= NQ && !LAR_WAIT(17, true, wait_or_abort(bar_qempty + slot * 8, (uint32_t)((seg / NQ - 1) & 1), abort_flag))) return false;
             const int unit = u0 + seg;
             const bool closes = (long long)(unit + 1) * T <= t_end;  // the segment holds the unit's last tile
             const bool with_kv = a.fused && closes;
@@ -267,6 +287,7 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
             if (lane < n_tiles) describe(lane, y_n, r, t);
             rt_n = r | (t << 8);
         }
+        LAR_STAMP(1);
         int stage = 0;
         uint32_t empty_parity = 1;
         for (int j0 = 0; j0 < n_tiles; j0 += 32) {
@@ -282,8 +303,12 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
                 const int yi = __shfl_sync(0xffffffffu, y, i), rti = __shfl_sync(0xffffffffu, rt, i);
                 if (lane == 0 && ok) {
                     const int ri = rti & 0xff;
-                    if (dep_waited && (j == 0 || (rti >> 8) == 0)) ok = issue_inputs(q_next++);
-                    if (ok) ok = wait_or_abort(bar_empty + stage * 8, empty_parity, abort_flag);
+                    if (dep_waited && (j == 0 || (rti >> 8) == 0)) {
+                        // first tile of a segment: its inputs and those of the next segment must be on their way
+                        const int seg_now = (int)((t_begin + j) / T) - u0;
+                        while (ok && q_next < n_segs && q_next <= seg_now + 1) ok = issue_inputs(q_next++);
+                    }
+                    if (ok) ok = LAR_WAIT(16, true, wait_or_abort(bar_empty + stage * 8, empty_parity, abort_flag));
                     if (ok) {
                         const uint32_t bar = bar_full + stage * 8, dst = ring + (uint32_t)stage * TR::STAGE_BYTES;
                         if (ri > 0) {
@@ -304,10 +329,11 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
                     // the ring is full of this layer's cache; everything else depends on the preceding kernel
                     grid_dep_wait();
                     grid_dep_launch();
+                    LAR_STAMP(2);
                     dep_waited = true;
                     if (lane == 0) {
                         const int seg_now = (int)((t_begin + j) / T) - u0;
-                        while (ok && q_next <= seg_now) ok = issue_inputs(q_next++);
+                        while (ok && q_next < n_segs && q_next <= seg_now + 1) ok = issue_inputs(q_next++);
                     }
                 }
             }
@@ -316,6 +342,7 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
             grid_dep_wait();
             grid_dep_launch();
         }
+        LAR_STAMP(3);
         if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
     } else if (warp <= W) {
         // =========================================================================== consumers
@@ -335,7 +362,8 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
 
             // ---- Q fragments (A operand): row qrow = head, 16 columns per k-step; heads >= G are zero rows
             const int qs = seg % NQ;
-            ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag);
+            ok = LAR_WAIT(18, cw == 0, wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag));
+            if (cw == 0 && seg == 0) LAR_STAMP(4);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             uint32_t qa0[TR::KSTEPS], qa2[TR::KSTEPS];
             {
@@ -354,13 +382,15 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
             if (lane == 0) mbar_arrive(bar_qempty + qs * 8);
 
             float m = -INFINITY, l = 0.f;  // head qrow; l is this thread's share of the row sum
-            float o[TR::NTILES][4];
+            // O^T: o[t][0], o[t][1] = heads 2 quad, 2 quad + 1 at d = 16 t + qrow; o[t][2], o[t][3] at d + 8
+            float o[TR::KSTEPS][4];
 #pragma unroll
-            for (int t = 0; t < TR::NTILES; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
+            for (int t = 0; t < TR::KSTEPS; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
 
             for (; j < je; j += W) {
                 const int s = stage;
-                ok = wait_or_abort(bar_full + s * 8, full_parity, abort_flag);
+                ok = LAR_WAIT(19, cw == 0, wait_or_abort(bar_full + s * 8, full_parity, abort_flag));
+                if (j == 0) LAR_STAMP(5);
                 if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
                 stage += W;
                 if (stage >= NS) {
@@ -404,10 +434,12 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
                     l = l * corr + (pr[0] + pr[1]) + (pr[2] + pr[3]);
                     m = m_new;
                     if (__any_sync(0xffffffffu, corr != 1.f)) {
+                        // the accumulator columns of this thread belong to heads 2 quad and 2 quad + 1
+                        const float ca = __shfl_sync(0xffffffffu, corr, 8 * quad), cb = __shfl_sync(0xffffffffu, corr, 8 * quad + 4);
 #pragma unroll
-                        for (int t = 0; t < TR::NTILES; ++t) { o[t][0] *= corr; o[t][1] *= corr; }
+                        for (int t = 0; t < TR::KSTEPS; ++t) { o[t][0] *= ca; o[t][1] *= cb; o[t][2] *= ca; o[t][3] *= cb; }
                     }
-                    const uint32_t pa0 = pack_bf16(pr[0], pr[1]), pa2 = pack_bf16(pr[2], pr[3]);
+                    const uint32_t pb0 = pack_bf16(pr[0], pr[1]), pb1 = pack_bf16(pr[2], pr[3]);  // P^T as B operand
                     // a short box leaves the lines behind its V rows unwritten: their weight is 0, but
                     // 0 * (stale NaN) is not
                     if (box_rows < kGranule) {
@@ -418,13 +450,12 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
                         }
                         __syncwarp();
                     }
-                    // O[head][d] += P V
+                    // O^T[d][head] += V^T[d][key] P^T[key][head]
 #pragma unroll
-                    for (int t = 0; t < TR::NTILES / 2; ++t) {
-                        uint32_t b[4];
-                        ldmatrix_x4_trans(St + tile_off<D>(box_rows + (lane & 7) + 8 * ((lane >> 3) & 1), 2 * t + (lane >> 4)), b);
-                        mma_bf16(o[2 * t], pa0, 0u, pa2, 0u, b[0], b[1]);
-                        mma_bf16(o[2 * t + 1], pa0, 0u, pa2, 0u, b[2], b[3]);
+                    for (int t = 0; t < TR::KSTEPS; ++t) {
+                        uint32_t af[4];
+                        ldmatrix_x4_trans(St + tile_off<D>(box_rows + (lane & 7) + 8 * (lane >> 4), 2 * t + ((lane >> 3) & 1)), af);
+                        mma_bf16(o[t], af[0], af[1], af[2], af[3], pb0, pb1);
                     }
                     if (box_rows < kGranule) fence_proxy_async_smem();  // zero-fill before the next TMA write
                 }
@@ -436,24 +467,36 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
             // ---- this warp's partial of the segment -> shared memory
             const int buf = seg & 1;
             if (seg >= 2) {
-                ok = wait_or_abort(bar_pempty + buf * 8, (uint32_t)((seg / 2 - 1) & 1), abort_flag);
+                ok = LAR_WAIT(20, cw == 0, wait_or_abort(bar_pempty + buf * 8, (uint32_t)((seg / 2 - 1) & 1), abort_flag));
                 if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             }
             l += __shfl_xor_sync(0xffffffffu, l, 1);
             l += __shfl_xor_sync(0xffffffffu, l, 2);
-            if (qrow < G) {
-                float* dstp = pbuf + buf * pbuf_floats + (cw * G + qrow) * PS;
+            {
+                float* wp = pbuf + buf * pbuf_floats + cw * G * PS;
+                if (2 * quad < G) {
 #pragma unroll
-                for (int t = 0; t < TR::NTILES; ++t)
-                    *reinterpret_cast<float2*>(dstp + 8 * t + 2 * quad) = make_float2(o[t][0], o[t][1]);
-                if (quad == 0) {
-                    dstp[D] = m;
-                    dstp[D + 1] = l;
+                    for (int t = 0; t < TR::KSTEPS; ++t) {
+                        wp[2 * quad * PS + 16 * t + qrow] = o[t][0];
+                        wp[2 * quad * PS + 16 * t + 8 + qrow] = o[t][2];
+                    }
+                }
+                if (2 * quad + 1 < G) {
+#pragma unroll
+                    for (int t = 0; t < TR::KSTEPS; ++t) {
+                        wp[(2 * quad + 1) * PS + 16 * t + qrow] = o[t][1];
+                        wp[(2 * quad + 1) * PS + 16 * t + 8 + qrow] = o[t][3];
+                    }
+                }
+                if (qrow < G && quad == 0) {
+                    wp[qrow * PS + D] = m;
+                    wp[qrow * PS + D + 1] = l;
                 }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_pfull + buf * 8);
         }
+        if (cw == 0) LAR_STAMP(6);
         if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
     } else {
         // =========================================================================== epilogue
@@ -481,7 +524,7 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
             const bool opens = ub >= t_begin, closes = ub + T <= t_end;
             const int qs = seg % NQ, buf = seg & 1;
             closing_loads(seg + 1, page_nxt, dev_len_nxt);
-            ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag);
+            ok = LAR_WAIT(21, true, wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag));
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             const unsigned char* Qs = qring_ptr + qs * QENT;
             const uint16_t* Q16 = reinterpret_cast<const uint16_t*>(Qs);
@@ -550,7 +593,8 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
             if (lane == 0) mbar_arrive(bar_qempty + qs * 8);
 
             // ---- merge the consumers' partials (+ the step's token)
-            ok = wait_or_abort(bar_pfull + buf * 8, (uint32_t)((seg / 2) & 1), abort_flag);
+            ok = LAR_WAIT(22, true, wait_or_abort(bar_pfull + buf * 8, (uint32_t)((seg / 2) & 1), abort_flag));
+            if (seg == 0) LAR_STAMP(7);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             const float* pb = pbuf + buf * pbuf_floats;
             float Mg[G], Lg[G], Og[G][PER];
@@ -611,23 +655,52 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
                 ticket = __shfl_sync(0xffffffffu, ticket, 0);
                 if (ticket == n_parts - 1) {
                     __threadfence();
+                    // All loads of a pass are independent of one another (no load waits for an exponential),
+                    // so the pass costs one trip to L2, not one per part.
                     const float* all = a.partials + (size_t)unit * a.max_seg * G * PS;
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
+                        // lane s holds (m, l) of part s (+32, ...): M = max m, L = sum l 2^(m - M)
                         float M = -INFINITY;
-                        for (int s = 0; s < n_parts; ++s) M = fmaxf(M, __ldcg(all + (s * G + g) * PS + D));
+                        for (int s0 = lane; s0 < n_parts; s0 += 32) M = fmaxf(M, __ldcg(all + (s0 * G + g) * PS + D));
+#pragma unroll
+                        for (int off = 16; off >= 1; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
                         float L = 0.f, O[PER];
 #pragma unroll
                         for (int i = 0; i < PER; ++i) O[i] = 0.f;
-                        for (int s = 0; s < n_parts; ++s) {
-                            const float* ps = all + (s * G + g) * PS;
-                            const float f = exp2_or_zero(__ldcg(ps + D), M);
-                            if (f != 0.f) {
-                                L = fmaf(__ldcg(ps + D + 1), f, L);
+                        for (int base = 0; base < n_parts; base += 32) {
+                            const int cnt = n_parts - base < 32 ? n_parts - base : 32;
+                            float f_own = 0.f;
+                            if (lane < cnt) {
+                                const float* ps = all + ((base + lane) * G + g) * PS;
+                                f_own = exp2_or_zero(__ldcg(ps + D), M);
+                                L = fmaf(__ldcg(ps + D + 1), f_own, L);
+                            }
+                            int s0 = 0;
+                            for (; s0 + 4 <= cnt; s0 += 4) {
+                                float v[4][PER];
 #pragma unroll
-                                for (int i = 0; i < PER; ++i) O[i] = fmaf(__ldcg(ps + lane + 32 * i), f, O[i]);
+                                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                                    for (int i = 0; i < PER; ++i) v[u][i] = __ldcg(all + ((base + s0 + u) * G + g) * PS + lane + 32 * i);
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    const float f = __shfl_sync(0xffffffffu, f_own, s0 + u);
+#pragma unroll
+                                    for (int i = 0; i < PER; ++i) O[i] = fmaf(v[u][i], f, O[i]);
+                                }
+                            }
+                            for (; s0 < cnt; ++s0) {
+                                float v[PER];
+#pragma unroll
+                                for (int i = 0; i < PER; ++i) v[i] = __ldcg(all + ((base + s0) * G + g) * PS + lane + 32 * i);
+                                const float f = __shfl_sync(0xffffffffu, f_own, s0);
+#pragma unroll
+                                for (int i = 0; i < PER; ++i) O[i] = fmaf(v[i], f, O[i]);
                             }
                         }
+#pragma unroll
+                        for (int off = 16; off >= 1; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
                         const float inv = L > 0.f ? 1.f / L : 0.f;
 #pragma unroll
                         for (int i = 0; i < PER; ++i)
@@ -637,6 +710,7 @@ __global__ void __launch_bounds__(192, 2) decode_stream_kernel(const StreamArgs 
                 }
             }
         }
+        LAR_STAMP(8);
         if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
     }
 

@@ -67,7 +67,7 @@ bool derive(const lar_config_t* c, Derived& d) {
     if (c->page_tokens != 0 && c->page_tokens != 16 && c->page_tokens != 32 && c->page_tokens != 64) return false;
     if (c->kv_splits != 0 && c->kv_splits != 1 && c->kv_splits != 2 && c->kv_splits != 4 && c->kv_splits != 8) return false;
     if (c->dtype == LAR_BF16) {
-        if (c->warps_per_cta < 0 || c->warps_per_cta > 4 || c->stages < 0 || c->stages == 1 || c->stages > 32) return false;
+        if (c->warps_per_cta < 0 || c->warps_per_cta > 6 || c->stages < 0 || c->stages == 1 || c->stages > 32) return false;
     } else {
         if (c->warps_per_cta < 0 || c->warps_per_cta > 8 || c->stages < 0 || c->stages > 4) return false;
     }
@@ -707,6 +707,18 @@ lar_status_t lar_cache_get_state(lar_cache_t* c, int layer, int32_t* lens, int32
     }
     return LAR_OK;
 }
+
+#ifdef LAR_TRACE
+// Trace builds only: copy the in-kernel timeline of the decode kernel (32 words per CTA) to the host and clear it.
+lar_status_t lar_debug_trace_read(unsigned long long* host_out, int n_ctas) {
+    if (!host_out || n_ctas < 1 || n_ctas > 1024) return LAR_ERR_INVALID_ARG;
+    LAR_CUDA(cudaDeviceSynchronize());
+    LAR_CUDA(cudaMemcpyFromSymbol(host_out, lar::lar_trace_buf, sizeof(unsigned long long) * 32 * (size_t)n_ctas));
+    static unsigned long long zeros[1024 * 32];
+    LAR_CUDA(cudaMemcpyToSymbol(lar::lar_trace_buf, zeros, sizeof(zeros)));
+    return LAR_OK;
+}
+#endif
 
 lar_status_t lar_cache_poll_device_status(lar_cache_t* c, uint32_t* bits_out, void* stream) {
     if (!c) return LAR_ERR_INVALID_ARG;
