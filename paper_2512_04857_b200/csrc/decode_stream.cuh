@@ -109,6 +109,7 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {
 }
 
 // ---- shared-memory plan of decode_stream_kernel (host and device agree through these) -------------
+constexpr int kMaxConsumers = 6;  // consumer warps per CTA at most
 __host__ __device__ constexpr int stream_q_slots(int G) { return G <= 2 ? 8 : 4; }
 __host__ __device__ constexpr int stream_q_entry_bytes(int D, int G) { return ((G + 2) * D * 2 + 127) / 128 * 128; }
 __host__ __device__ constexpr int stream_fixed_smem_bytes(int D, int G, int W) {
@@ -595,31 +596,39 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
             // ---- merge the consumers' partials (+ the step's token)
             ok = LAR_WAIT(22, true, wait_or_abort(bar_pfull + buf * 8, (uint32_t)((seg / 2) & 1), abort_flag));
             if (seg == 0) LAR_STAMP(7);
+            LAR_STAMP(9);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             const float* pb = pbuf + buf * pbuf_floats;
+            // branch-free and unrolled over the (at most kMaxConsumers) consumer warps, so that the shared-memory
+            // loads of all heads are in flight together
             float Mg[G], Lg[G], Og[G][PER];
 #pragma unroll
             for (int g = 0; g < G; ++g) {
+                float mw[kMaxConsumers], fw[kMaxConsumers];
                 float M = s_new[g];
-                for (int w = 0; w < W; ++w) M = fmaxf(M, pb[(w * G + g) * PS + D]);
+#pragma unroll
+                for (int w = 0; w < kMaxConsumers; ++w) {
+                    mw[w] = w < W ? pb[(w * G + g) * PS + D] : -INFINITY;
+                    M = fmaxf(M, mw[w]);
+                }
                 const float f_new = exp2_or_zero(s_new[g], M);
                 float L = f_new;
 #pragma unroll
                 for (int i = 0; i < PER; ++i) Og[g][i] = v_new[i] * f_new;
-                for (int w = 0; w < W; ++w) {
-                    const float* pw = pb + (w * G + g) * PS;
-                    const float f = exp2_or_zero(pw[D], M);
-                    if (f != 0.f) {
-                        L = fmaf(pw[D + 1], f, L);
 #pragma unroll
-                        for (int i = 0; i < PER; ++i) Og[g][i] = fmaf(pw[lane + 32 * i], f, Og[g][i]);
-                    }
+                for (int w = 0; w < kMaxConsumers; ++w) {
+                    const float* pw = pb + ((w < W ? w : 0) * G + g) * PS;
+                    fw[w] = exp2_or_zero(mw[w], M);
+                    L = fmaf(pw[D + 1], fw[w], L);
+#pragma unroll
+                    for (int i = 0; i < PER; ++i) Og[g][i] = fmaf(pw[lane + 32 * i], fw[w], Og[g][i]);
                 }
                 Mg[g] = M;
                 Lg[g] = L;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_pempty + buf * 8);
+            LAR_STAMP(10);
 
             if (opens && closes) {
                 // the whole unit lies in this CTA
@@ -653,60 +662,59 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
                 int ticket = 0;
                 if (lane == 0) ticket = atomicAdd(a.tickets + unit, 1);
                 ticket = __shfl_sync(0xffffffffu, ticket, 0);
+                LAR_STAMP(11);
                 if (ticket == n_parts - 1) {
                     __threadfence();
-                    // All loads of a pass are independent of one another (no load waits for an exponential),
-                    // so the pass costs one trip to L2, not one per part.
+                    // Heads in groups of GC, parts in pairs: the loads of a pair (m, l and the o row of every head
+                    // of the group) are independent of one another and of any exponential, so a pair costs one
+                    // trip to L2; the pairs are folded in online-softmax fashion.
                     const float* all = a.partials + (size_t)unit * a.max_seg * G * PS;
+                    constexpr int GC = G < 4 ? G : 4;
 #pragma unroll
-                    for (int g = 0; g < G; ++g) {
-                        // lane s holds (m, l) of part s (+32, ...): M = max m, L = sum l 2^(m - M)
-                        float M = -INFINITY;
-                        for (int s0 = lane; s0 < n_parts; s0 += 32) M = fmaxf(M, __ldcg(all + (s0 * G + g) * PS + D));
+                    for (int g0 = 0; g0 < G; g0 += GC) {
+                        float M[GC], L[GC], O[GC][PER];
 #pragma unroll
-                        for (int off = 16; off >= 1; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
-                        float L = 0.f, O[PER];
+                        for (int c = 0; c < GC; ++c) {
+                            M[c] = -INFINITY;
+                            L[c] = 0.f;
 #pragma unroll
-                        for (int i = 0; i < PER; ++i) O[i] = 0.f;
-                        for (int base = 0; base < n_parts; base += 32) {
-                            const int cnt = n_parts - base < 32 ? n_parts - base : 32;
-                            float f_own = 0.f;
-                            if (lane < cnt) {
-                                const float* ps = all + ((base + lane) * G + g) * PS;
-                                f_own = exp2_or_zero(__ldcg(ps + D), M);
-                                L = fmaf(__ldcg(ps + D + 1), f_own, L);
-                            }
-                            int s0 = 0;
-                            for (; s0 + 4 <= cnt; s0 += 4) {
-                                float v[4][PER];
+                            for (int i = 0; i < PER; ++i) O[c][i] = 0.f;
+                        }
+                        for (int s0 = 0; s0 < n_parts; s0 += 2) {
+                            float mv[2][GC], lv2[2][GC], ov[2][GC][PER];
 #pragma unroll
-                                for (int u = 0; u < 4; ++u)
+                            for (int u = 0; u < 2; ++u) {
+                                const bool have = s0 + u < n_parts;
+                                const float* ps = all + ((have ? s0 + u : s0) * G + g0) * PS;
 #pragma unroll
-                                    for (int i = 0; i < PER; ++i) v[u][i] = __ldcg(all + ((base + s0 + u) * G + g) * PS + lane + 32 * i);
+                                for (int c = 0; c < GC; ++c) {
+                                    mv[u][c] = __ldcg(ps + c * PS + D);
+                                    lv2[u][c] = __ldcg(ps + c * PS + D + 1);
 #pragma unroll
-                                for (int u = 0; u < 4; ++u) {
-                                    const float f = __shfl_sync(0xffffffffu, f_own, s0 + u);
-#pragma unroll
-                                    for (int i = 0; i < PER; ++i) O[i] = fmaf(v[u][i], f, O[i]);
+                                    for (int i = 0; i < PER; ++i) ov[u][c][i] = __ldcg(ps + c * PS + lane + 32 * i);
+                                    if (!have) mv[u][c] = -INFINITY;
                                 }
                             }
-                            for (; s0 < cnt; ++s0) {
-                                float v[PER];
 #pragma unroll
-                                for (int i = 0; i < PER; ++i) v[i] = __ldcg(all + ((base + s0) * G + g) * PS + lane + 32 * i);
-                                const float f = __shfl_sync(0xffffffffu, f_own, s0);
+                            for (int c = 0; c < GC; ++c) {
+                                const float Mn = fmaxf(M[c], fmaxf(mv[0][c], mv[1][c]));
+                                const float f_old = exp2_or_zero(M[c], Mn), f0 = exp2_or_zero(mv[0][c], Mn), f1 = exp2_or_zero(mv[1][c], Mn);
+                                L[c] = L[c] * f_old + lv2[0][c] * f0 + lv2[1][c] * f1;
 #pragma unroll
-                                for (int i = 0; i < PER; ++i) O[i] = fmaf(v[i], f, O[i]);
+                                for (int i = 0; i < PER; ++i) O[c][i] = O[c][i] * f_old + ov[0][c][i] * f0 + ov[1][c][i] * f1;
+                                M[c] = Mn;
                             }
                         }
 #pragma unroll
-                        for (int off = 16; off >= 1; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
-                        const float inv = L > 0.f ? 1.f / L : 0.f;
+                        for (int c = 0; c < GC; ++c) {
+                            const float inv = L[c] > 0.f ? 1.f / L[c] : 0.f;
 #pragma unroll
-                        for (int i = 0; i < PER; ++i)
-                            outp[((size_t)unit * G + g) * D + lane + 32 * i] = __float2bfloat16_rn(O[i] * inv);
+                            for (int i = 0; i < PER; ++i)
+                                outp[((size_t)unit * G + g0 + c) * D + lane + 32 * i] = __float2bfloat16_rn(O[c][i] * inv);
+                        }
                     }
                     if (lane == 0) a.tickets[unit] = 0;
+                    LAR_STAMP(12);
                 }
             }
         }
