@@ -81,7 +81,7 @@ typedef struct lar_config {
     int32_t recent_lines;  /* r >= 1: the last r lines are never evicted (Sec. 3.3) */
     int32_t budget_lines;  /* B / n (Sec. 3.3 "Cache Budget"); >= n_lines selects the full-cache path */
     float softmax_scale;   /* 0 selects 1/sqrt(head_dim) (Eq. 2) */
-    int32_t page_tokens;   /* tokens per physical page: 16, 32 or 64; 0 selects 16 */
+    int32_t page_tokens;   /* tokens per physical page: fp32 16, 32 or 64 (0 selects 16); bf16 32 or 64 (0 selects 32) */
     uint32_t flags;        /* LAR_FLAG_* */
     int32_t kv_splits;     /* fp32 only: CTAs (one thread-block cluster) per unit in decode: 0 auto, else 1,2,4,8 */
     int32_t warps_per_cta; /* decode warps: bf16 consumer warps per CTA, 0 auto, else 1..6;

@@ -1,7 +1,7 @@
 // bf16 decode attention (Eq. 2-3) as one persistent, warp-specialised streaming kernel per layer-step,
 // fused with the append of the step's token (Eq. 4) and the guide-queue push (Eq. 8).
 //
-// Work decomposition.  The live rows of every unit = (sequence, KV head) are cut into 16-row tiles;
+// Work decomposition.  The live rows of every unit = (sequence, KV head) are cut into 32-row tiles;
 // all tiles of the layer form one list (unit-major) that is dealt out in contiguous ranges to the CTAs
 // of the grid (one CTA per SM).  Where whole units can be dealt out evenly enough the ranges end on unit
 // boundaries; otherwise they are equal in tiles, so that every SM streams the same number of bytes
@@ -40,8 +40,10 @@ namespace lar {
 struct TensorMaps {
     // 3-D maps over {head_dim, pool rows of all layers, {K pool, V pool}}: one copy brings the K rows and
     // the V rows of a tile; box = 64 elements x 4 (i + 1) rows x 2
-    CUtensorMap kv[4];
+    CUtensorMap kv[8];
 };
+
+constexpr int kStreamTile = 32;  // rows of K (and of V) per tile of the streaming kernel; a tile lies inside one page
 
 struct StreamArgs {
     LayerView lv;
@@ -94,7 +96,7 @@ template <int D>
 struct MmaTraits {
     static constexpr int ROW_BYTES = D * 2;
     static constexpr int HALVES = D / 64;                  // 128-byte column blocks per row
-    static constexpr int HALF_BYTES = 2 * kGranule * 128;  // one swizzled block: [K rows | V rows][64 elements]
+    static constexpr int HALF_BYTES = 2 * kStreamTile * 128;  // one swizzled block: [K rows | V rows][64 elements]
     static constexpr int STAGE_BYTES = HALVES * HALF_BYTES;
     static constexpr int KSTEPS = D / 16;
     static constexpr int NTILES = D / 8;
@@ -119,7 +121,7 @@ __host__ __device__ constexpr int stream_fixed_smem_bytes(int D, int G, int W) {
            + (2 * stream_q_slots(G) + 4) * 8 + 16;            // query / partial barriers, abort flag
 }
 __host__ __device__ constexpr int stream_smem_bytes(int D, int G, int W, int NS) {
-    return stream_fixed_smem_bytes(D, G, W) + NS * (2 * (D / 64) * kGranule * 128 + 16);  // stage + its 2 barriers
+    return stream_fixed_smem_bytes(D, G, W) + NS * (2 * (D / 64) * kStreamTile * 128 + 16);  // stage + its 2 barriers
 }
 
 // Wait on an mbarrier phase; gives up (and raises the CTA-wide abort flag) after ~1 s of SM clocks or as
@@ -222,7 +224,7 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
 
     // ---- the layer's tile list and this CTA's range of it
     const int len = a.len, n_tok = a.n_tok;
-    const int T = len > 0 ? (len + kGranule - 1) / kGranule : 1;  // an empty cache is one tile of 0 rows
+    const int T = len > 0 ? (len + kStreamTile - 1) / kStreamTile : 1;  // an empty cache is one tile of 0 rows
     const long long total = (long long)a.n_units * T;
     long long t_begin = 0, t_end = 0;
     int Pe;  // CTAs that get work: every range is non-empty
@@ -254,8 +256,8 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
             const long long t = t_begin + jj;
             const int unit = (int)(t / T);
             tile = (int)(t - (long long)unit * T);
-            const int row0 = tile * kGranule;
-            rows = len - row0 < kGranule ? len - row0 : kGranule;
+            const int row0 = tile * kStreamTile;
+            rows = len - row0 < kStreamTile ? len - row0 : kStreamTile;
             if (rows > 0) {
                 const int page = __ldg(&lv.page_table[unit * lv.pages_per_unit + row0 / lv.page_tokens]);
                 y = a.pool_row_base + page * lv.page_tokens + row0 % lv.page_tokens;
@@ -399,40 +401,39 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
                     full_parity ^= 1u;
                 }
                 const int tile = (int)(t_begin + j - ub);
-                const int rows = len - tile * kGranule < kGranule ? len - tile * kGranule : kGranule;
+                const int rows = len - tile * kStreamTile < kStreamTile ? len - tile * kStreamTile : kStreamTile;
                 const uint32_t St = ring + (uint32_t)s * TR::STAGE_BYTES;
                 if (rows > 0) {
                     const int box_rows = (rows + 3) & ~3;  // K rows are lines 0.., V rows lines box_rows.. of a block
-                    // S[head][key] for the 16 keys of the tile: two n-tiles of 8 keys, two accumulators each
-                    float sc[2][2][4];
+                    // S[head][key] for the 32 keys of the tile: four n-tiles of 8 keys
+                    float sc[4][4];
 #pragma unroll
-                    for (int jn = 0; jn < 2; ++jn) {
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) sc[jn][0][e] = sc[jn][1][e] = 0.f;
+                    for (int jn = 0; jn < 4; ++jn) {
+                        sc[jn][0] = sc[jn][1] = sc[jn][2] = sc[jn][3] = 0.f;
 #pragma unroll
                         for (int i = 0; i < TR::KSTEPS / 2; ++i) {
                             uint32_t b[4];
                             ldmatrix_x4(St + tile_off<D>(8 * jn + (lane & 7), 4 * i + (lane >> 3)), b);
-                            mma_bf16(sc[jn][0], qa0[2 * i], 0u, qa2[2 * i], 0u, b[0], b[1]);
-                            mma_bf16(sc[jn][1], qa0[2 * i + 1], 0u, qa2[2 * i + 1], 0u, b[2], b[3]);
+                            mma_bf16(sc[jn], qa0[2 * i], 0u, qa2[2 * i], 0u, b[0], b[1]);
+                            mma_bf16(sc[jn], qa0[2 * i + 1], 0u, qa2[2 * i + 1], 0u, b[2], b[3]);
                         }
                     }
-                    // online softmax over the keys this thread holds: 2*quad, 2*quad+1 (+8)
-                    float sv[4];
+                    // online softmax over the keys this thread holds: 8 jn + 2 quad, + 1
+                    float sv[8];
 #pragma unroll
-                    for (int jn = 0; jn < 2; ++jn) {
-                        sv[2 * jn + 0] = (8 * jn + 2 * quad + 0 < rows) ? (sc[jn][0][0] + sc[jn][1][0]) * a.scale_log2 : -INFINITY;
-                        sv[2 * jn + 1] = (8 * jn + 2 * quad + 1 < rows) ? (sc[jn][0][1] + sc[jn][1][1]) * a.scale_log2 : -INFINITY;
+                    for (int jn = 0; jn < 4; ++jn) {
+                        sv[2 * jn + 0] = (8 * jn + 2 * quad + 0 < rows) ? sc[jn][0] * a.scale_log2 : -INFINITY;
+                        sv[2 * jn + 1] = (8 * jn + 2 * quad + 1 < rows) ? sc[jn][1] * a.scale_log2 : -INFINITY;
                     }
-                    float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+                    float mx = fmaxf(fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3])), fmaxf(fmaxf(sv[4], sv[5]), fmaxf(sv[6], sv[7])));
                     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
                     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
                     const float m_new = fmaxf(m, mx);
                     const float corr = exp2f(m - m_new);
-                    float pr[4];
+                    float pr[8];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) pr[i] = exp2f(sv[i] - m_new);
-                    l = l * corr + (pr[0] + pr[1]) + (pr[2] + pr[3]);
+                    for (int i = 0; i < 8; ++i) pr[i] = exp2f(sv[i] - m_new);
+                    l = l * corr + ((pr[0] + pr[1]) + (pr[2] + pr[3])) + ((pr[4] + pr[5]) + (pr[6] + pr[7]));
                     m = m_new;
                     if (__any_sync(0xffffffffu, corr != 1.f)) {
                         // the accumulator columns of this thread belong to heads 2 quad and 2 quad + 1
@@ -440,11 +441,13 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
 #pragma unroll
                         for (int t = 0; t < TR::KSTEPS; ++t) { o[t][0] *= ca; o[t][1] *= cb; o[t][2] *= ca; o[t][3] *= cb; }
                     }
-                    const uint32_t pb0 = pack_bf16(pr[0], pr[1]), pb1 = pack_bf16(pr[2], pr[3]);  // P^T as B operand
+                    // P^T as B operand: keys 0-15 and keys 16-31
+                    const uint32_t pb00 = pack_bf16(pr[0], pr[1]), pb01 = pack_bf16(pr[2], pr[3]);
+                    const uint32_t pb10 = pack_bf16(pr[4], pr[5]), pb11 = pack_bf16(pr[6], pr[7]);
                     // a short box leaves the lines behind its V rows unwritten: their weight is 0, but
                     // 0 * (stale NaN) is not
-                    if (box_rows < kGranule) {
-                        const int n16 = (kGranule - box_rows) * 8;  // 16-byte chunks per block
+                    if (box_rows < kStreamTile) {
+                        const int n16 = (kStreamTile - box_rows) * 8;  // 16-byte chunks per block
                         for (int i = lane; i < n16 * TR::HALVES; i += 32) {
                             const int h = i / n16, c = i - h * n16;
                             asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(St + h * TR::HALF_BYTES + 2 * box_rows * 128 + c * 16), "r"(0u) : "memory");
@@ -456,9 +459,11 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
                     for (int t = 0; t < TR::KSTEPS; ++t) {
                         uint32_t af[4];
                         ldmatrix_x4_trans(St + tile_off<D>(box_rows + (lane & 7) + 8 * (lane >> 4), 2 * t + ((lane >> 3) & 1)), af);
-                        mma_bf16(o[t], af[0], af[1], af[2], af[3], pb0, pb1);
+                        mma_bf16(o[t], af[0], af[1], af[2], af[3], pb00, pb01);
+                        ldmatrix_x4_trans(St + tile_off<D>(box_rows + 16 + (lane & 7) + 8 * (lane >> 4), 2 * t + ((lane >> 3) & 1)), af);
+                        mma_bf16(o[t], af[0], af[1], af[2], af[3], pb10, pb11);
                     }
-                    if (box_rows < kGranule) fence_proxy_async_smem();  // zero-fill before the next TMA write
+                    if (box_rows < kStreamTile) fence_proxy_async_smem();  // zero-fill before the next TMA write
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_empty + s * 8);

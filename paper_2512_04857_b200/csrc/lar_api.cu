@@ -65,6 +65,7 @@ bool derive(const lar_config_t* c, Derived& d) {
     if (c->cond_len < 0 || c->line_width < 1 || c->n_lines < 1 || c->anchor_len < 0) return false;
     if (c->recent_lines < 1 || c->budget_lines < 1) return false;
     if (c->page_tokens != 0 && c->page_tokens != 16 && c->page_tokens != 32 && c->page_tokens != 64) return false;
+    if (c->dtype == LAR_BF16 && c->page_tokens == 16) return false;  // a 32-row tile of the bf16 decode kernel lies in one page
     if (c->kv_splits != 0 && c->kv_splits != 1 && c->kv_splits != 2 && c->kv_splits != 4 && c->kv_splits != 8) return false;
     if (c->dtype == LAR_BF16) {
         if (c->warps_per_cta < 0 || c->warps_per_cta > 6 || c->stages < 0 || c->stages == 1 || c->stages > 32) return false;
@@ -88,7 +89,7 @@ bool derive(const lar_config_t* c, Derived& d) {
     d.elt = c->dtype == LAR_BF16 ? 2 : 4;
     d.row_bytes = c->head_dim * d.elt;
     d.cap = c->cond_len + d.B;
-    d.P = c->page_tokens ? c->page_tokens : 16;
+    d.P = c->page_tokens ? c->page_tokens : (c->dtype == LAR_BF16 ? 32 : 16);
     d.ppu = (d.cap + d.P - 1) / d.P;
     d.cap_pad = d.ppu * d.P;
     d.mid_pad = (int)align_up((size_t)(d.M > 0 ? d.M : 1), 4);
@@ -101,7 +102,7 @@ bool derive(const lar_config_t* c, Derived& d) {
         if (c->flags & LAR_FLAG_TILE_RANGES) d.unit_ranges = 0;
     }
     d.max_seg = 1;
-    const int t_max = (d.cap + lar::kGranule - 1) / lar::kGranule;
+    const int t_max = (d.cap + lar::kStreamTile - 1) / lar::kStreamTile;
     for (int T = 1; T <= t_max; ++T) {
         const long long chunk = (long long)d.units * T / d.ctas;
         long long b = chunk >= 1 ? (T + chunk - 1) / chunk + 1 : T;
@@ -154,7 +155,7 @@ void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
         int NS = c->stages;
         if (NS == 0) {
             const int budget = 110 * 1024;
-            const int stage = 2 * (c->head_dim / 64) * lar::kGranule * 128 + 16;
+            const int stage = 2 * (c->head_dim / 64) * lar::kStreamTile * 128 + 16;
             const int fixed = c->head_dim == 64 ? lar::stream_fixed_smem_bytes(64, d.group, W) : lar::stream_fixed_smem_bytes(128, d.group, W);
             NS = (budget - fixed) / stage;
             if (NS > 32) NS = 32;
@@ -292,7 +293,7 @@ lar_status_t make_tensor_maps(lar_cache* c) {
     const cuuint64_t gdim[3] = {(cuuint64_t)c->cfg.head_dim, (cuuint64_t)c->rows_per_layer * (cuuint64_t)c->cfg.n_layers, 2};
     const cuuint64_t gstride[2] = {(cuuint64_t)c->d.row_bytes, (cuuint64_t)(c->L.off_vpool - c->L.off_kpool)};
     const cuuint32_t estr[3] = {1, 1, 1};
-    for (int h = 0; h < 4; ++h) {
+    for (int h = 0; h < 8; ++h) {
         const cuuint32_t box[3] = {64, (cuuint32_t)(4 * (h + 1)), 2};
         CUresult r = encode(&c->tmaps.kv[h], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, c->slab + c->L.off_kpool, gdim, gstride, box,
                             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
