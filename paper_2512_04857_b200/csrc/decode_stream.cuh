@@ -113,11 +113,12 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {
 // ---- shared-memory plan of decode_stream_kernel (host and device agree through these) -------------
 constexpr int kMaxConsumers = 6;  // consumer warps per CTA at most
 __host__ __device__ constexpr int stream_q_slots(int G) { return G <= 2 ? 8 : 4; }
+__host__ __device__ constexpr int stream_partial_bufs(int G) { return G <= 2 ? 2 : 1; }  // partial buffers per CTA
 __host__ __device__ constexpr int stream_q_entry_bytes(int D, int G) { return ((G + 2) * D * 2 + 127) / 128 * 128; }
 __host__ __device__ constexpr int stream_fixed_smem_bytes(int D, int G, int W) {
     return 1024                                               // slack: the ring starts on a 1024-byte boundary
            + stream_q_slots(G) * stream_q_entry_bytes(D, G)   // query ring
-           + 2 * (W + 1) * G * (D + 2) * 4                    // two partial buffers
+           + stream_partial_bufs(G) * (W + 1) * G * (D + 2) * 4  // partial buffers
            + (2 * stream_q_slots(G) + 4) * 8 + 16;            // query / partial barriers, abort flag
 }
 __host__ __device__ constexpr int stream_smem_bytes(int D, int G, int W, int NS) {
@@ -177,6 +178,7 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
     using TR = MmaTraits<D>;
     using T16 = __nv_bfloat16;
     constexpr int NQ = stream_q_slots(G);
+    constexpr int NPB = stream_partial_bufs(G);
     constexpr int QENT = stream_q_entry_bytes(D, G);
     constexpr int PS = D + 2;  // floats per (warp, head) partial: o[D], m, l
     constexpr int PER = D / 32;
@@ -194,7 +196,7 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
     const uint32_t qring = smem_u32(qring_ptr);
     float* pbuf = reinterpret_cast<float*>(qring_ptr + NQ * QENT);
     const int pbuf_floats = (W + 1) * G * PS;
-    unsigned char* bars_ptr = reinterpret_cast<unsigned char*>(pbuf + 2 * pbuf_floats);
+    unsigned char* bars_ptr = reinterpret_cast<unsigned char*>(pbuf + NPB * pbuf_floats);
     const uint32_t bars = smem_u32(bars_ptr);
     const uint32_t bar_full = bars, bar_empty = bars + NS * 8;
     const uint32_t bar_qfull = bars + 2 * NS * 8, bar_qempty = bar_qfull + NQ * 8;
@@ -471,9 +473,9 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
             if (!ok) break;
 
             // ---- this warp's partial of the segment -> shared memory
-            const int buf = seg & 1;
-            if (seg >= 2) {
-                ok = LAR_WAIT(20, cw == 0, wait_or_abort(bar_pempty + buf * 8, (uint32_t)((seg / 2 - 1) & 1), abort_flag));
+            const int buf = seg % NPB;
+            if (seg >= NPB) {
+                ok = LAR_WAIT(20, cw == 0, wait_or_abort(bar_pempty + buf * 8, (uint32_t)((seg / NPB - 1) & 1), abort_flag));
                 if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             }
             l += __shfl_xor_sync(0xffffffffu, l, 1);
@@ -528,7 +530,7 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
             const int unit = u0 + seg;
             const long long ub = (long long)unit * T;
             const bool opens = ub >= t_begin, closes = ub + T <= t_end;
-            const int qs = seg % NQ, buf = seg & 1;
+            const int qs = seg % NQ, buf = seg % NPB;
             closing_loads(seg + 1, page_nxt, dev_len_nxt);
             ok = LAR_WAIT(21, true, wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag));
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
@@ -599,7 +601,7 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
             if (lane == 0) mbar_arrive(bar_qempty + qs * 8);
 
             // ---- merge the consumers' partials (+ the step's token)
-            ok = LAR_WAIT(22, true, wait_or_abort(bar_pfull + buf * 8, (uint32_t)((seg / 2) & 1), abort_flag));
+            ok = LAR_WAIT(22, true, wait_or_abort(bar_pfull + buf * 8, (uint32_t)((seg / NPB) & 1), abort_flag));
             if (seg == 0) LAR_STAMP(7);
             LAR_STAMP(9);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }

@@ -151,10 +151,10 @@ void make_layout(const lar_config_t* c, const Derived& d, Layout& L) {
 // fp32: one cluster of X CTAs per unit, W warps per CTA, NS stages per warp.
 void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
     if (c->dtype == LAR_BF16) {
-        const int W = c->warps_per_cta ? c->warps_per_cta : 4;
+        const int W = c->warps_per_cta ? c->warps_per_cta : 3;
         int NS = c->stages;
         if (NS == 0) {
-            const int budget = 110 * 1024;
+            const int budget = 113 * 1024;  // two CTAs (+ 1 KB each of system use) share the 228 KB of an SM
             const int stage = 2 * (c->head_dim / 64) * lar::kStreamTile * 128 + 16;
             const int fixed = c->head_dim == 64 ? lar::stream_fixed_smem_bytes(64, d.group, W) : lar::stream_fixed_smem_bytes(128, d.group, W);
             NS = (budget - fixed) / stage;
