@@ -169,6 +169,8 @@ class Runner:
         flags = lar.LAR_FLAG_NO_HOST_CHECKS | flags_extra
         if not args.no_pdl:
             flags |= lar.LAR_FLAG_PDL
+        if args.tile_ranges:
+            flags |= lar.LAR_FLAG_TILE_RANGES
         self.cfg = lar.config_from_workload(w, flags=flags, kv_splits=args.kv_splits, warps_per_cta=args.warps,
                                             stages=args.stages, page_tokens=args.page_tokens, decode_ctas=args.ctas)
         self.cache = lar.Cache(self.cfg, device=str(dev))
@@ -487,6 +489,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling / small cases)")
     ap.add_argument("--eager", action="store_true", help="plain stream launches instead of CUDA graphs (profiling)")
     ap.add_argument("--no-pdl", action="store_true")
+    ap.add_argument("--tile-ranges", action="store_true", help="deal 32-row tiles, not whole units, to the decode CTAs")
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

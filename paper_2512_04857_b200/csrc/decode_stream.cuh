@@ -113,7 +113,7 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {
 // ---- shared-memory plan of decode_stream_kernel (host and device agree through these) -------------
 constexpr int kMaxConsumers = 6;  // consumer warps per CTA at most
 __host__ __device__ constexpr int stream_q_slots(int G) { return G <= 2 ? 8 : 4; }
-__host__ __device__ constexpr int stream_partial_bufs(int G) { return G <= 2 ? 2 : 1; }  // partial buffers per CTA
+__host__ __device__ constexpr int stream_partial_bufs(int) { return 2; }  // partial buffers per CTA
 __host__ __device__ constexpr int stream_q_entry_bytes(int D, int G) { return ((G + 2) * D * 2 + 127) / 128 * 128; }
 __host__ __device__ constexpr int stream_fixed_smem_bytes(int D, int G, int W) {
     return 1024                                               // slack: the ring starts on a 1024-byte boundary

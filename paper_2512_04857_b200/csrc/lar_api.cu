@@ -93,14 +93,17 @@ bool derive(const lar_config_t* c, Derived& d) {
     d.ppu = (d.cap + d.P - 1) / d.P;
     d.cap_pad = d.ppu * d.P;
     d.mid_pad = (int)align_up((size_t)(d.M > 0 ? d.M : 1), 4);
-    // A unit of T tiles is cut into at most ceil(T / floor(U T / P)) + 1 segments (never more than T or P).
+    // Grid of the persistent bf16 decode kernel.  With fewer units than SMs every unit gets the same whole
+    // number of CTAs (none is idle, merges stay k-way).  Whole units per CTA wherever that keeps the busiest
+    // CTA within 25 % of the average (nothing to merge across CTAs); equal tile ranges otherwise.
     d.ctas = c->decode_ctas ? c->decode_ctas : kDefaultDecodeCtas;
-    // Whole units per CTA when that leaves at most ~6 % of imbalance: no unit is cut, nothing to merge.
+    if (!c->decode_ctas && d.units < d.ctas) d.ctas = d.units * (d.ctas / d.units);
     {
         const long long per = ((long long)d.units + d.ctas - 1) / d.ctas;
-        d.unit_ranges = (d.units >= d.ctas && per * d.ctas * 100 <= (long long)d.units * 106) ? 1 : 0;
+        d.unit_ranges = (d.units >= d.ctas && (long long)d.units * 10 >= per * d.ctas * 8) ? 1 : 0;
         if (c->flags & LAR_FLAG_TILE_RANGES) d.unit_ranges = 0;
     }
+    // A unit of T tiles is cut into at most ceil(T / floor(U T / P)) + 1 segments (never more than T or P).
     d.max_seg = 1;
     const int t_max = (d.cap + lar::kStreamTile - 1) / lar::kStreamTile;
     for (int T = 1; T <= t_max; ++T) {
@@ -162,6 +165,7 @@ void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
         }
         // a stage must always be read by the same consumer warp: ring depth = a multiple of W
         NS = NS / W * W;
+        if (c->stages == 0 && NS < 2 * W) NS = 2 * W;  // rather a deep ring than two CTAs per SM
         if (NS < W) NS = W;
         if (NS < 2) NS = 2;
         p.kv_splits = 1;
