@@ -95,42 +95,40 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------------
-def cpu_baseline(w, budget_s: float = 12.0, seed_units: int = 8):
-    """Time the CPU oracle, as it stands, on a bounded sample of the workload's independent units."""
+def cpu_baseline(w, budget_s: float = 12.0, sample_units: int = 256):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload's independent units.
+
+    The sample is `sample_units` whole (layer, sequence, kv-head) units (every token of the generation, line-end
+    evictions included); the same sample is run repeatedly until about `budget_s` seconds of oracle time have
+    passed (the oracle's cost does not depend on the values)."""
     import numpy as np
     from oracle import lar_oracle as O
     from paper_2512_04857_b200 import workloads as W
-    cores = os.cpu_count() or 1
     cfg = O.cfg_from_workload(w)
-
-    def sample(n_units, first):
-        us = []
-        for i in range(n_units):
-            j = first + i
-            layer = j % w.n_layers
-            s = (j // w.n_layers) % w.batch
-            h = (j // (w.n_layers * w.batch)) % w.n_kv_heads
-            us.append(W.gen_unit(w, layer, s, h))
-        st = lambda key: np.stack([u[key].numpy() for u in us])
-        return st("q"), st("k"), st("v"), st("kc"), st("vc")
-
-    ins = sample(seed_units, 0)
-    t0 = time.perf_counter()
-    _, _, thr = O.run_units(cfg, *ins, want_out=False, want_kept=False)
-    t_probe = time.perf_counter() - t0
-    per_unit = t_probe / seed_units
-    n_units = int(min(max(seed_units, budget_s / max(per_unit, 1e-6)), 64 * cores, w.n_layers * w.n_units))
-    n_units = max(cores, (n_units // cores) * cores)
-    ins = sample(n_units, seed_units)
-    t0 = time.perf_counter()
-    _, _, thr = O.run_units(cfg, *ins, want_out=True, want_kept=True)
-    dt = time.perf_counter() - t0
-    units_per_image = w.n_layers * w.n_units / w.images
-    value = (n_units / units_per_image) * w.n_visual / dt
+    total_units = w.n_layers * w.n_units
+    out_bytes_per_unit = w.n_visual * w.group * w.head_dim * 8      # the oracle returns fp64 outputs
+    n_units = max(1, min(sample_units, total_units, (512 << 20) // out_bytes_per_unit))
+    us = []
+    for j in range(n_units):
+        layer = j % w.n_layers
+        s = (j // w.n_layers) % w.batch
+        h = (j // (w.n_layers * w.batch)) % w.n_kv_heads
+        us.append(W.gen_unit(w, layer, s, h))
+    st = lambda key: np.stack([u[key].numpy() for u in us])
+    ins = (st("q"), st("k"), st("v"), st("kc"), st("vc"))
+    O.run_units(cfg, *[x[:8] for x in ins], want_out=False, want_kept=False)   # page the library in
+    passes, dt, thr = 0, 0.0, 1
+    while dt < budget_s and passes < 1000:
+        t0 = time.perf_counter()
+        _, _, thr = O.run_units(cfg, *ins, want_out=True, want_kept=True)
+        dt += time.perf_counter() - t0
+        passes += 1
+    units_per_image = total_units / w.images
+    value = (n_units * passes / units_per_image) * w.n_visual / dt
     return {"value": value, "unit": UNIT, "cores": int(thr), "kind": "oracle",
-            "sample": f"{n_units} of {w.n_layers * w.n_units} independent (layer, sequence, kv-head) units of "
-                      f"'{w.name}', whole generation ({w.n_visual} tokens, line-end evictions), {dt:.1f} s",
-            "seconds": dt, "units": n_units}
+            "sample": f"{n_units} of {total_units} independent (layer, sequence, kv-head) units of '{w.name}', whole "
+                      f"generation ({w.n_visual} tokens, line-end evictions), {passes} passes, {dt:.1f} s of oracle time",
+            "seconds": dt, "units": n_units * passes}
 
 
 def run_reference(args):
@@ -226,7 +224,7 @@ class Runner:
                                 self.cache.append_kv(layer, self.kc[layer], self.vc[layer], self.w.cond_len)
                     self._enqueue_decode(line)
                 gb = None
-                if line < self.w.n_lines - 1:
+                if line < self.w.n_lines - 1 and not self.w.is_full_cache:
                     gb = torch.cuda.CUDAGraph()
                     with torch.cuda.graph(gb, stream=s):
                         self._enqueue_line_end(line)
@@ -409,7 +407,7 @@ def run_ours(args):
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": w.name, "layers": w.n_layers, "sequences": w.batch, "images": w.images,
                        "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
                        "storage": w.dtype, "prefix": w.cond_len, "grid": f"{w.n_lines}x{w.line_width}",
@@ -421,7 +419,7 @@ def run_ours(args):
                        "plan": main["plan"], "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
             "clocks": main["clocks"],
             "gpu_launches": main["launches"] * args.steps,
-            "roofline": {"bound": "hbm", "kernel": "decode_kernel (fused append + decode attention)",
+            "roofline": {"bound": "hbm", "kernel": "decode_stream_kernel (fused append + decode attention)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_kind": f"of {peak_kind} copy bandwidth",
                          "frac_of_8TBs": achieved / 8000.0,
