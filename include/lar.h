@@ -189,6 +189,29 @@ uint64_t lar_cache_launch_count(const lar_cache_t* c);
 /* The plan a cache was created with. */
 lar_status_t lar_cache_get_plan(const lar_cache_t* c, lar_plan_t* plan_out);
 
+/* Decode attention over dense K/V without any scratch buffer from the caller (the paper has no counterpart of this
+ * call; it exists for callers that cannot allocate).  The other entry points keep their split-KV partials in the
+ * caller's slab.  A caller that only owns its q / K / V / out tensors and may not call cudaMalloc at this point --
+ * code running inside a framework's memory-pool "no allocation" region, a serving loop that has already handed all
+ * free memory to its KV-cache manager, a plug-in that was given pointers and nothing else -- has no slab to offer.
+ * For them the partials live in a file-scope device array of the library: 8 MiB on every GPU that loads the
+ * library, held until the process exits.
+ *
+ *   out[u][g] = softmax(q[u][g] K[u]^T scale) V[u]      (Eq. 2 per unit u and query head g of its group)
+ *   q, out : device, bf16, [n_units, group, head_dim]      k, v : device, bf16, [n_units, len, head_dim], dense
+ *   group 1..8, head_dim 64 or 128, len >= 1, softmax_scale 0 selects 1/sqrt(head_dim).
+ *
+ * Limits: n_units <= 16384 (one ticket per unit), otherwise LAR_ERR_CAPACITY and nothing is launched; the number of
+ * key ranges per unit (at most 8) is reduced until n_units * ranges * group * (head_dim + 2) * 4 bytes fit into the
+ * array, so larger problems run with fewer CTAs rather than fail.
+ * The call enqueues one memset (the tickets of the units it uses must start at zero; the array keeps whatever the
+ * previous call left) and one kernel on `stream`, and calls no allocating routine.  The first call on a device looks
+ * the array's device address up (cudaGetSymbolAddress, with that device current): make that first call outside any
+ * stream capture.  All calls on a device share the one array: two calls whose kernels may overlap on the GPU
+ * (different streams, no dependency) race on it -- order them. */
+lar_status_t lar_attend_dense_noalloc(const void* q, const void* k, const void* v, void* out, int n_units, int group,
+                                      int head_dim, int len, float softmax_scale, void* stream);
+
 const char* lar_status_str(lar_status_t s);
 int lar_last_cuda_error(void); /* cudaError_t of the last failed runtime call in this thread, 0 if none */
 

@@ -14,6 +14,7 @@
 #include "decode_attn.cuh"
 #include "decode_stream.cuh"
 #include "line_end.cuh"
+#include "attend_noalloc.cuh"
 
 namespace {
 
@@ -733,6 +734,30 @@ lar_status_t lar_cache_poll_device_status(lar_cache_t* c, uint32_t* bits_out, vo
     if (bits) LAR_CUDA(cudaMemset(c->slab + c->L.off_status, 0, sizeof(bits)));
     if (bits_out) *bits_out = bits;
     return bits ? LAR_ERR_DEVICE_CHECK : LAR_OK;
+}
+
+lar_status_t lar_attend_dense_noalloc(const void* q, const void* k, const void* v, void* out, int n_units, int group,
+                                      int head_dim, int len, float softmax_scale, void* stream) {
+    if (!q || !k || !v || !out || n_units < 1 || len < 1) return LAR_ERR_INVALID_ARG;
+    if (group < 1 || group > 8 || !(head_dim == 64 || head_dim == 128)) return LAR_ERR_INVALID_ARG;
+    if (!(softmax_scale >= 0.f) || !isfinite(softmax_scale)) return LAR_ERR_INVALID_ARG;
+    if (n_units > lar::kStaticMaxUnits) return LAR_ERR_CAPACITY;  // one ticket per unit in the static array
+    unsigned char* scratch = nullptr;
+    LAR_CUDA(lar::static_scratch_address(&scratch));
+    const int splits = lar::static_scratch_splits(n_units, group, head_dim, len);
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
+    cudaStream_t s = (cudaStream_t)stream;
+    // the array keeps what the last call left: the tickets of this call must start at zero
+    LAR_CUDA(cudaMemsetAsync(scratch, 0, (size_t)n_units * sizeof(int), s));
+    const dim3 grid((unsigned)(n_units * splits));
+    if (head_dim == 64)
+        lar::attend_dense_kernel<64><<<grid, 128, 0, s>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
+                                                          (__nv_bfloat16*)out, scratch, group, len, splits, scale * 1.4426950408889634f);
+    else
+        lar::attend_dense_kernel<128><<<grid, 128, 0, s>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
+                                                           (__nv_bfloat16*)out, scratch, group, len, splits, scale * 1.4426950408889634f);
+    LAR_CUDA(cudaGetLastError());
+    return LAR_OK;
 }
 
 }  // extern "C"

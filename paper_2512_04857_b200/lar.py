@@ -74,6 +74,7 @@ def lib():
         "lar_cache_set_host_checks": (C.c_int, [vp, ip]),
         "lar_cache_launch_count": (C.c_uint64, [vp]),
         "lar_cache_get_plan": (C.c_int, [vp, planp]),
+        "lar_attend_dense_noalloc": (C.c_int, [vp, vp, vp, vp, ip, ip, ip, ip, C.c_float, vp]),
         "lar_status_str": (C.c_char_p, [C.c_int]),
         "lar_last_cuda_error": (C.c_int, []),
     }
@@ -193,6 +194,12 @@ def lar_cache_get_plan(cache) -> lar_plan_t:
     plan = lar_plan_t()
     _chk(lib().lar_cache_get_plan(cache, C.byref(plan)), "lar_cache_get_plan")
     return plan
+
+
+def lar_attend_dense_noalloc(q, k, v, out, n_units, group, head_dim, length, softmax_scale=0.0, stream=None):
+    """Decode attention over dense bf16 K/V; the split-KV scratch is a static device array of the library."""
+    _chk(lib().lar_attend_dense_noalloc(_ptr(q), _ptr(k), _ptr(v), _ptr(out), n_units, group, head_dim, length,
+                                        float(softmax_scale), stream), "lar_attend_dense_noalloc")
 
 
 class Cache:
