@@ -212,7 +212,8 @@ lar_status_t plan_query_impl(const lar_config_t* cfg, lar_plan_t* out, Derived* 
     p.compressing = d.compressing;
     choose_plan(cfg, d, p);
     p.line_end_smem_bytes =
-        d.compressing ? lar::line_end_smem_bytes(d.row_bytes, cfg->head_dim, d.M, d.M - cfg->line_width + cfg->recent_lines * cfg->line_width, 8) : 0;
+        d.compressing ? lar::line_end_smem_bytes(d.row_bytes, cfg->head_dim, d.M, d.M - cfg->line_width + cfg->recent_lines * cfg->line_width, 8,
+                                                 cfg->line_width * d.group, cfg->dtype == LAR_BF16 ? 1 : 0) : 0;
     p.slab_bytes = L.total;
     p.scratch_bytes = (L.off_tickets + L.tickets_bytes) - L.off_partials;
     if (p.decode_smem_bytes > 227 * 1024 || p.line_end_smem_bytes > 227 * 1024) return LAR_ERR_INVALID_ARG;

@@ -3,7 +3,8 @@
 // compact K, V and the index map in place.
 #pragma once
 #include "common.cuh"
-#include "decode_attn.cuh"  // warp_max / warp_sum
+#include "decode_attn.cuh"    // warp_max / warp_sum
+#include "decode_stream.cuh"  // ldmatrix / mma wrappers
 
 namespace lar {
 
@@ -41,18 +42,97 @@ __global__ void __launch_bounds__(128) append_kernel(const LayerView lv, const T
 }
 
 // ------------------------------------------------------------------------------------- line end
-// Shared memory of line_end_kernel (bytes), M mid keys, W warps.
-__host__ __device__ inline int line_end_smem_bytes(int row_bytes, int D, int M, int total_rows, int warps) {
-    int b = M * (row_bytes + 16);          // mid keys, rows padded by one chunk against bank conflicts
-    b += warps * (D + 2 * M) * 4;          // per warp: query row (fp32), logits row, score accumulator
+// Shared memory of line_end_kernel (bytes): M mid keys, nq = n * G guide rows, W warps.
+// bf16 (tensor-core scoring): the guide rows are staged next to the keys; fp32: per-warp row buffers.
+__host__ __device__ inline int line_end_smem_bytes(int row_bytes, int D, int M, int total_rows, int warps, int nq, int is_bf16) {
+    int b = ((M + 7) / 8 * 8) * (row_bytes + 16);  // mid keys (whole 8-key tiles), rows padded by one chunk against bank conflicts
+    if (is_bf16)
+        b += ((nq + 15) / 16 * 16) * (row_bytes + 16) + M * 4;  // guide rows (whole 16-row tiles), column sums
+    else
+        b += warps * (D + 2 * M) * 4;      // per warp: query row (fp32), logits row, score accumulator
     b += M * 4;                            // final scores
     b += ((M + 3) / 4) * 4;                // keep flags
     b += total_rows * 4;                   // source slot of every surviving row
     return (b + 15) / 16 * 16 + 16;
 }
 
-// One CTA per unit.  CUDA-core version: every lane owns the keys m = lane, lane + 32, ... and computes
-// whole dot products against a query row broadcast from shared memory.
+// Eq. 9 on tensor cores (bf16).  kmid: [M8][KROW] keys, qg: [nq16][KROW] guide rows (both staged, rows of KROW
+// bytes), colsum: [M] zeroed.  Every warp takes 16-row blocks of guide rows; a block's logits against all keys
+// are formed twice with mma.sync m16n8k16 -- once for the row maxima and sums, once more to add the normalised
+// probabilities into the column sums -- which is cheaper than keeping a [16][M] tile of logits anywhere.
+template <int D>
+__device__ __forceinline__ void score_mma(const unsigned char* kmid, const unsigned char* qg, float* colsum, int M, int nq,
+                                          float scale_log2, int warp, int lane, int W) {
+    constexpr int KROW = D * 2 + 16;
+    constexpr int KSTEPS = D / 16;
+    const int quad = lane & 3, grow = lane >> 2;
+    const int n_tiles = (M + 7) / 8;
+    const uint32_t kbase = smem_u32(kmid), qbase = smem_u32(qg);
+    for (int rb = warp; rb * 16 < nq; rb += W) {
+        uint32_t a[KSTEPS][4];
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks)
+            ldmatrix_x4(qbase + (uint32_t)((rb * 16 + (lane & 15)) * KROW + (2 * ks + (lane >> 4)) * 16), a[ks]);
+        auto logits = [&](int nt, float (&c)[4]) {
+            c[0] = c[1] = c[2] = c[3] = 0.f;
+#pragma unroll
+            for (int i = 0; i < KSTEPS / 2; ++i) {
+                uint32_t b[4];
+                ldmatrix_x4(kbase + (uint32_t)((nt * 8 + (lane & 7)) * KROW + (4 * i + (lane >> 3)) * 16), b);
+                mma_bf16(c, a[2 * i][0], a[2 * i][1], a[2 * i][2], a[2 * i][3], b[0], b[1]);
+                mma_bf16(c, a[2 * i + 1][0], a[2 * i + 1][1], a[2 * i + 1][2], a[2 * i + 1][3], b[2], b[3]);
+            }
+            const int key = nt * 8 + 2 * quad;
+            c[0] = key < M ? c[0] * scale_log2 : -INFINITY;
+            c[2] = key < M ? c[2] * scale_log2 : -INFINITY;
+            c[1] = key + 1 < M ? c[1] * scale_log2 : -INFINITY;
+            c[3] = key + 1 < M ? c[3] * scale_log2 : -INFINITY;
+        };
+        // pass 1: maximum and sum of every row (rows grow and grow + 8 of the block; this thread's columns first)
+        float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+        for (int nt = 0; nt < n_tiles; ++nt) {
+            float c[4];
+            logits(nt, c);
+            const float n0 = fmaxf(m0, fmaxf(c[0], c[1])), n1 = fmaxf(m1, fmaxf(c[2], c[3]));
+            l0 = l0 * exp2f(m0 - n0) + exp2f(c[0] - n0) + exp2f(c[1] - n0);
+            l1 = l1 * exp2f(m1 - n1) + exp2f(c[2] - n1) + exp2f(c[3] - n1);
+            m0 = n0;
+            m1 = n1;
+        }
+#pragma unroll
+        for (int off = 1; off <= 2; off <<= 1) {
+            const float om0 = __shfl_xor_sync(0xffffffffu, m0, off), ol0 = __shfl_xor_sync(0xffffffffu, l0, off);
+            const float om1 = __shfl_xor_sync(0xffffffffu, m1, off), ol1 = __shfl_xor_sync(0xffffffffu, l1, off);
+            const float n0 = fmaxf(m0, om0), n1 = fmaxf(m1, om1);
+            l0 = l0 * exp2f(m0 - n0) + ol0 * exp2f(om0 - n0);
+            l1 = l1 * exp2f(m1 - n1) + ol1 * exp2f(om1 - n1);
+            m0 = n0;
+            m1 = n1;
+        }
+        // rows beyond the queue (the last block may be ragged) carry no weight
+        const float w0 = rb * 16 + grow < nq ? 1.f / l0 : 0.f, w1 = rb * 16 + grow + 8 < nq ? 1.f / l1 : 0.f;
+        // pass 2: probabilities, summed over the block's rows, into the column sums
+        for (int nt = 0; nt < n_tiles; ++nt) {
+            float c[4];
+            logits(nt, c);
+            float v0 = (w0 != 0.f ? exp2f(c[0] - m0) * w0 : 0.f) + (w1 != 0.f ? exp2f(c[2] - m1) * w1 : 0.f);
+            float v1 = (w0 != 0.f ? exp2f(c[1] - m0) * w0 : 0.f) + (w1 != 0.f ? exp2f(c[3] - m1) * w1 : 0.f);
+#pragma unroll
+            for (int off = 4; off <= 16; off <<= 1) {
+                v0 += __shfl_xor_sync(0xffffffffu, v0, off);
+                v1 += __shfl_xor_sync(0xffffffffu, v1, off);
+            }
+            if (grow == 0) {
+                const int key = nt * 8 + 2 * quad;
+                if (key < M) atomicAdd(colsum + key, v0);
+                if (key + 1 < M) atomicAdd(colsum + key + 1, v1);
+            }
+        }
+    }
+}
+
+// One CTA per unit.  Scoring: bf16 on tensor cores (score_mma); fp32 on CUDA cores, where every lane owns the keys
+// m = lane, lane + 32, ... and computes whole dot products against a query row broadcast from shared memory.
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(256) line_end_kernel(const LayerView lv, float scale_log2) {
     constexpr int EPL = Elt<T>::kPerChunk;
@@ -80,71 +160,97 @@ __global__ void __launch_bounds__(256) line_end_kernel(const LayerView lv, float
     const int total_rows = n_keep + n_rec;                    // rows behind the anchor after compaction
     const int nq = n * G;
 
+    constexpr bool kMma = sizeof(T) == 2;  // bf16: tensor-core scoring; fp32: CUDA cores
+    const int M8 = (M + 7) / 8 * 8, nq16 = (nq + 15) / 16 * 16;
     unsigned char* kmid = smem;
-    float* wbuf = reinterpret_cast<float*>(smem + (size_t)M * KROW);
-    float* qrow = wbuf + warp * (D + 2 * M);
-    float* logit = qrow + D;
-    float* sacc = logit + M;
-    float* S = wbuf + W * (D + 2 * M);
+    unsigned char* after_k = smem + (size_t)M8 * KROW;
+    unsigned char* qg = after_k;                                                // [nq16][KROW]   (bf16)
+    float* colsum = reinterpret_cast<float*>(after_k + (size_t)nq16 * KROW);    // [M]            (bf16)
+    float* wbuf = reinterpret_cast<float*>(after_k);                            // [W][D + 2 M]   (fp32)
+    float* S = kMma ? colsum + M : wbuf + W * (D + 2 * M);
     unsigned char* keep = reinterpret_cast<unsigned char*>(S + M);
     int* srcmap = reinterpret_cast<int*>(keep + ((M + 3) / 4) * 4);
 
-    // ---- stage the mid keys
-    for (int idx = tid; idx < M * CHUNKS; idx += blockDim.x) {
+    // ---- stage the mid keys (rows of the last, ragged 8-key tile are cleared)
+    for (int idx = tid; idx < M8 * CHUNKS; idx += blockDim.x) {
         const int r = idx / CHUNKS, c = idx - r * CHUNKS;
-        const size_t off = row_offset(lv, unit, mid0 + r, ROW_BYTES) + c * 16;
-        *reinterpret_cast<uint4*>(kmid + r * KROW + c * 16) = *reinterpret_cast<const uint4*>(lv.k_pool + off);
+        uint4 val = make_uint4(0u, 0u, 0u, 0u);
+        if (r < M) val = *reinterpret_cast<const uint4*>(lv.k_pool + row_offset(lv, unit, mid0 + r, ROW_BYTES) + c * 16);
+        *reinterpret_cast<uint4*>(kmid + r * KROW + c * 16) = val;
     }
-    for (int mm = lane; mm < M; mm += 32) sacc[mm] = 0.f;
-    __syncthreads();
-
-    // ---- Eq. 9: every guide row is soft-maxed over the M mid keys; rows are summed per key
     const T* gq = reinterpret_cast<const T*>(lv.guide) + (size_t)unit * nq * D;
-    for (int j = warp; j < nq; j += W) {
-        for (int c = lane; c < CHUNKS; c += 32) {
-            const uint4 raw = *reinterpret_cast<const uint4*>(gq + (size_t)j * D + c * EPL);
-            float f[EPL];
-            Elt<T>::unpack(raw, f);
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) qrow[c * EPL + e] = f[e] * scale_log2;
+    if constexpr (kMma) {
+        // ---- Eq. 9 on tensor cores: stage the guide rows, clear the column sums
+        for (int idx = tid; idx < nq16 * CHUNKS; idx += blockDim.x) {
+            const int r = idx / CHUNKS, c = idx - r * CHUNKS;
+            uint4 val = make_uint4(0u, 0u, 0u, 0u);
+            if (r < nq) val = *reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(gq) + (size_t)r * ROW_BYTES + c * 16);
+            *reinterpret_cast<uint4*>(qg + r * KROW + c * 16) = val;
         }
-        __syncwarp();
-        float mx = -INFINITY;
-        for (int mm = lane; mm < M; mm += 32) {
-            const unsigned char* kr = kmid + mm * KROW;
-            float acc = 0.f;
-#pragma unroll 4
-            for (int c = 0; c < CHUNKS; ++c) {
-                float kf[EPL];
-                Elt<T>::unpack(*reinterpret_cast<const uint4*>(kr + c * 16), kf);
+        for (int mm = tid; mm < M; mm += blockDim.x) colsum[mm] = 0.f;
+        __syncthreads();
+        score_mma<D>(kmid, qg, colsum, M, nq, scale_log2, warp, lane, W);
+        __syncthreads();
+        const float inv_nq = 1.f / (float)nq;
+        for (int mm = tid; mm < M; mm += blockDim.x) {
+            const float sc = colsum[mm] * inv_nq;
+            S[mm] = sc;
+            lv.scores[(size_t)unit * lv.mid_pad + mm] = sc;
+        }
+        __syncthreads();
+    } else {
+        // ---- Eq. 9 on CUDA cores: every guide row is soft-maxed over the M mid keys; rows are summed per key
+        float* qrow = wbuf + warp * (D + 2 * M);
+        float* logit = qrow + D;
+        float* sacc = logit + M;
+        for (int mm = lane; mm < M; mm += 32) sacc[mm] = 0.f;
+        __syncthreads();
+        for (int j = warp; j < nq; j += W) {
+            for (int c = lane; c < CHUNKS; c += 32) {
+                const uint4 raw = *reinterpret_cast<const uint4*>(gq + (size_t)j * D + c * EPL);
+                float f[EPL];
+                Elt<T>::unpack(raw, f);
 #pragma unroll
-                for (int e = 0; e < EPL; ++e) acc = fmaf(qrow[c * EPL + e], kf[e], acc);
+                for (int e = 0; e < EPL; ++e) qrow[c * EPL + e] = f[e] * scale_log2;
             }
-            logit[mm] = acc;
-            mx = fmaxf(mx, acc);
+            __syncwarp();
+            float mx = -INFINITY;
+            for (int mm = lane; mm < M; mm += 32) {
+                const unsigned char* kr = kmid + mm * KROW;
+                float acc = 0.f;
+#pragma unroll 4
+                for (int c = 0; c < CHUNKS; ++c) {
+                    float kf[EPL];
+                    Elt<T>::unpack(*reinterpret_cast<const uint4*>(kr + c * 16), kf);
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) acc = fmaf(qrow[c * EPL + e], kf[e], acc);
+                }
+                logit[mm] = acc;
+                mx = fmaxf(mx, acc);
+            }
+            mx = warp_max(mx);
+            float sum = 0.f;
+            for (int mm = lane; mm < M; mm += 32) {
+                const float p = exp2f(logit[mm] - mx);
+                logit[mm] = p;
+                sum += p;
+            }
+            sum = warp_sum(sum);
+            const float inv = 1.f / sum;
+            for (int mm = lane; mm < M; mm += 32) sacc[mm] = fmaf(logit[mm], inv, sacc[mm]);
+            __syncwarp();
         }
-        mx = warp_max(mx);
-        float sum = 0.f;
-        for (int mm = lane; mm < M; mm += 32) {
-            const float p = exp2f(logit[mm] - mx);
-            logit[mm] = p;
-            sum += p;
+        __syncthreads();
+        const float inv_nq = 1.f / (float)nq;
+        for (int mm = tid; mm < M; mm += blockDim.x) {
+            float sc = 0.f;
+            for (int w = 0; w < W; ++w) sc += wbuf[w * (D + 2 * M) + D + M + mm];
+            sc *= inv_nq;
+            S[mm] = sc;
+            lv.scores[(size_t)unit * lv.mid_pad + mm] = sc;
         }
-        sum = warp_sum(sum);
-        const float inv = 1.f / sum;
-        for (int mm = lane; mm < M; mm += 32) sacc[mm] = fmaf(logit[mm], inv, sacc[mm]);
-        __syncwarp();
+        __syncthreads();
     }
-    __syncthreads();
-    const float inv_nq = 1.f / (float)nq;
-    for (int mm = tid; mm < M; mm += blockDim.x) {
-        float s = 0.f;
-        for (int w = 0; w < W; ++w) s += wbuf[w * (D + 2 * M) + D + M + mm];
-        s *= inv_nq;
-        S[mm] = s;
-        lv.scores[(size_t)unit * lv.mid_pad + mm] = s;
-    }
-    __syncthreads();
 
     // ---- Eq. 10: keep the M - n most salient; equal scores keep the lower slot (older token)
     for (int mm = tid; mm < M; mm += blockDim.x) {
