@@ -279,7 +279,7 @@ __global__ void __launch_bounds__(256) line_end_kernel(const LayerView lv, float
     __syncthreads();
 
     // rows move towards lower slots only (src >= dst); tiles ascending, load - barrier - store
-    constexpr int TILE_ROWS = 32;
+    constexpr int TILE_ROWS = 1024 / CHUNKS;  // 4 chunks of K and 4 of V per thread in flight (32 .. 128 rows)
     int* imap = lv.index_map + (size_t)unit * lv.cap_pad;
     for (int t0 = 0; t0 < total_rows; t0 += TILE_ROWS) {
         const int rows = min(TILE_ROWS, total_rows - t0);
