@@ -160,7 +160,7 @@ def run_reference(args):
 class Runner:
     """Device-resident inputs + per-line CUDA graphs of one workload."""
 
-    def __init__(self, w, dev, args, flags_extra=0):
+    def __init__(self, w, dev, args, flags_extra=0, input_lines=0):
         import torch
         from paper_2512_04857_b200 import lar, workloads as W
         self.torch, self.lar, self.w, self.dev = torch, lar, w, dev
@@ -174,9 +174,12 @@ class Runner:
         self.cache = lar.Cache(self.cfg, device=str(dev))
         L, S, Hq, Hkv, d, n, h = w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.line_width, w.n_lines
         dt = w.torch_dtype
-        self.q = torch.empty((h, n, L, S, Hq, d), dtype=dt, device=dev)
-        self.k = torch.empty((h, n, L, S, Hkv, d), dtype=dt, device=dev)
-        self.v = torch.empty((h, n, L, S, Hkv, d), dtype=dt, device=dev)
+        # distinct lines of inputs kept resident (all of them by default); throughput does not depend on the
+        # values, so the batch sweep reuses a few lines to bound memory
+        hl = self.input_lines = h if input_lines <= 0 else min(h, input_lines)
+        self.q = torch.empty((hl, n, L, S, Hq, d), dtype=dt, device=dev)
+        self.k = torch.empty((hl, n, L, S, Hkv, d), dtype=dt, device=dev)
+        self.v = torch.empty((hl, n, L, S, Hkv, d), dtype=dt, device=dev)
         self.kc = torch.empty((L, S, Hkv, max(w.cond_len, 1), d), dtype=dt, device=dev)
         self.vc = torch.empty_like(self.kc)
         self.out = torch.empty((n, L, S, Hq, d), dtype=dt, device=dev)
@@ -184,7 +187,7 @@ class Runner:
             if w.cond_len:
                 a, b = W.gen_prefix(w, layer, dev)
                 self.kc[layer], self.vc[layer] = a, b
-            for line in range(h):
+            for line in range(hl):
                 q, k, v = W.gen_tokens(w, layer, line * n, (line + 1) * n, dev)
                 self.q[line, :, layer], self.k[line, :, layer], self.v[line, :, layer] = q, k, v
         torch.cuda.synchronize(dev)
@@ -193,6 +196,7 @@ class Runner:
 
     def _enqueue_decode(self, line):
         w, c = self.w, self.cache
+        line = line % self.input_lines
         for t in range(w.line_width):
             for layer in range(w.n_layers):
                 c.decode_step(layer, self.q[line, t, layer], self.k[line, t, layer], self.v[line, t, layer],
@@ -374,8 +378,8 @@ def run_ours(args):
     if args.layers:
         w = w.scaled(n_layers=args.layers)
 
-    def bench_workload(wl, steps, warmup, sample_clocks):
-        r = Runner(wl, dev, args)
+    def bench_workload(wl, steps, warmup, sample_clocks, input_lines=0):
+        r = Runner(wl, dev, args, input_lines=input_lines)
         if args.eager:
             r.launches_per_generation = (wl.n_layers * (wl.n_visual + (1 if wl.cond_len else 0))
                                          + (0 if wl.is_full_cache else wl.n_layers * (wl.n_lines - 1)))
@@ -461,6 +465,22 @@ def run_ours(args):
             line["also"][name] = {"value": world * w2.images * w2.n_visual / (r2["ms_per_step"] * 1e-3), "unit": UNIT,
                                   "ms_per_step": r2["ms_per_step"], "roofline_achieved_gbs": ach,
                                   "roofline_frac": ach / peak, "frac_of_8TBs": ach / 8000.0, "plan": r2["plan"]}
+    # ---- batch sweep of one shape, compressed and full-cache (not the headline line)
+    if args.batch_sweep:
+        wb = W.WORKLOADS[args.sweep_workload]
+        line["batch_sweep"] = {"workload": wb.name, "inputs": "2 lines of inputs reused for every line", "points": []}
+        for b in [int(x) for x in args.batch_sweep.split(",")]:
+            w2 = wb.scaled(batch=2 * b, images=b)
+            rc = bench_workload(w2, 1, 1, False, input_lines=2)
+            ach = w2.kv_bytes_per_generation() / (rc["decode_ms_per_step"] * 1e-3) / 1e9
+            pt = {"images": b, "sequences": 2 * b, "value": world * b * w2.n_visual / (rc["ms_per_step"] * 1e-3),
+                  "ms_per_step": rc["ms_per_step"], "decode_launch_us": rc["decode_ms_per_step"] * 1e3 / (w2.n_visual * w2.n_layers),
+                  "roofline_achieved_gbs": ach, "roofline_frac": ach / peak, "frac_of_8TBs": ach / 8000.0, "plan": rc["plan"]}
+            if not args.no_full:
+                rf = bench_workload(w2.full_cache(), 1, 1, False, input_lines=2)
+                pt["full_cache_ms_per_step"] = rf["ms_per_step"]
+                pt["speedup_vs_full_cache"] = rf["ms_per_step"] / rc["ms_per_step"]
+            line["batch_sweep"]["points"].append(pt)
     # ---- CPU oracle on the host cores (rank 0, N = 1 only)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = {k: v for k, v in cpu_baseline(w).items() if k not in ("seconds", "units")}
@@ -479,6 +499,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="janus_pro_7b")
     ap.add_argument("--also", default="", help="comma-separated extra workloads reported under 'also'")
+    ap.add_argument("--batch-sweep", default="", help="comma-separated image counts: sweep the batch of --sweep-workload")
+    ap.add_argument("--sweep-workload", default="gqa_1024")
     ap.add_argument("--kv-splits", type=int, default=0)
     ap.add_argument("--warps", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)

@@ -62,11 +62,16 @@ struct StreamArgs {
     int pool_row_base;  // first pool row of this layer in the tensor maps
 };
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar, uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
-        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(policy)
         : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -293,6 +298,8 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
             rt_n = r | (t << 8);
         }
         LAR_STAMP(1);
+        // every cached row is read once per step: let it leave L2 first
+        const uint64_t pol_stream = l2_policy_evict_first();
         int stage = 0;
         uint32_t empty_parity = 1;
         for (int j0 = 0; j0 < n_tiles; j0 += 32) {
@@ -320,7 +327,7 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
                             const int hsel = (ri + 3) / 4 - 1;  // box of 4 * (hsel + 1) rows
                             mbar_expect_tx(bar, (uint32_t)(2 * 4 * (hsel + 1) * TR::ROW_BYTES));
 #pragma unroll
-                            for (int h = 0; h < TR::HALVES; ++h) tma_load_3d(dst + h * TR::HALF_BYTES, &tm.kv[hsel], h * 64, yi, 0, bar);
+                            for (int h = 0; h < TR::HALVES; ++h) tma_load_3d(dst + h * TR::HALF_BYTES, &tm.kv[hsel], h * 64, yi, 0, bar, pol_stream);
                         } else {
                             mbar_arrive(bar);  // nothing to fetch: release the consumer
                         }
