@@ -20,7 +20,7 @@ def nvcc_cmd(verbose: bool = False, trace: bool = False):
            "-Xcompiler", "-fPIC", "-shared",
            "-I", os.path.join(ROOT, "include"), "-o", OUT_TRACE if trace else OUT] + SOURCES
     if trace:
-        cmd[1:1] = ["-DLAR_TRACE"]
+        cmd[1:1] = ["-DLAR_TRACE"] + (["-DLAR_TRACE_STAMPS_ONLY"] if os.environ.get("LAR_TRACE_STAMPS_ONLY") else [])
     if verbose:
         cmd[1:1] = ["-Xptxas", "-v"]
     return cmd

@@ -30,6 +30,7 @@ struct LayerView {
     int pages_per_unit, page_tokens, cap, cap_pad, mid_pad;
     int cond_len, line_width, budget_tokens, anchor_len, recent_lines, compressing;
     int n_kv_heads, group;
+    int identity_pages;     // 1: unit u owns pages u * pages_per_unit ... in order (the table need not be read)
 };
 
 // ---------------------------------------------------------------------------------- PTX wrappers

@@ -157,8 +157,12 @@ __device__ __forceinline__ unsigned long long trace_now() {
     return t;
 }
 #define LAR_STAMP(slot) do { if ((threadIdx.x & 31) == 0) lar_trace_buf[blockIdx.x * 32 + (slot)] = trace_now(); } while (0)
+#ifdef LAR_TRACE_STAMPS_ONLY
+#define LAR_WAIT(slot, rec, call) (call)
+#else
 #define LAR_WAIT(slot, rec, call) [&]() { const long long t0__ = clock64(); const bool r__ = (call); \
     if ((rec) && (threadIdx.x & 31) == 0) atomicAdd(&lar_trace_buf[blockIdx.x * 32 + (slot)], (unsigned long long)(clock64() - t0__)); return r__; }()
+#endif
 #else
 #define LAR_STAMP(slot) do { } while (0)
 #define LAR_WAIT(slot, rec, call) (call)
@@ -266,7 +270,8 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
             const int row0 = tile * kStreamTile;
             rows = len - row0 < kStreamTile ? len - row0 : kStreamTile;
             if (rows > 0) {
-                const int page = __ldg(&lv.page_table[unit * lv.pages_per_unit + row0 / lv.page_tokens]);
+                const int pidx = unit * lv.pages_per_unit + row0 / lv.page_tokens;
+                const int page = lv.identity_pages ? pidx : __ldg(&lv.page_table[pidx]);
                 y = a.pool_row_base + page * lv.page_tokens + row0 % lv.page_tokens;
             } else {
                 y = 0;
@@ -527,7 +532,10 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
             page = 0;
             dev_len = len;
             if (sg < n_segs && (long long)(un + 1) * T <= t_end) {
-                if (a.fused && len < lv.cap) page = __ldg(&lv.page_table[un * lv.pages_per_unit + new_page_idx]);
+                if (a.fused && len < lv.cap) {
+                    const int pidx = un * lv.pages_per_unit + new_page_idx;
+                    page = lv.identity_pages ? pidx : __ldg(&lv.page_table[pidx]);
+                }
                 dev_len = __ldcg(&lv.state[un].len);
             }
         };

@@ -276,6 +276,7 @@ lar::LayerView view_of(const lar_cache* c, int layer) {
     v.compressing = d.compressing;
     v.n_kv_heads = c->cfg.n_kv_heads;
     v.group = d.group;
+    v.identity_pages = (c->cfg.flags & LAR_FLAG_SHUFFLE_PAGES) ? 0 : 1;
     return v;
 }
 
@@ -382,7 +383,10 @@ lar_status_t launch_append(lar_cache* c, int layer, const void* k, const void* v
 lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k, const void* v, void* out, int fused,
                            cudaStream_t s) {
     const bool pdl = (c->cfg.flags & LAR_FLAG_PDL) != 0;
-    const int prefetch = (pdl && c->last_layer != layer && c->last_layer >= 0) ? 1 : 0;
+    // Fetching cached K/V ahead of the dependency pays only if this launch's CTAs can move in beside the preceding
+    // kernel's (two per SM); otherwise they start when that kernel is done and want their inputs first.
+    const bool co_resident = c->cfg.dtype != LAR_BF16 || 2 * (c->plan.decode_smem_bytes + 1024) <= 228 * 1024;
+    const int prefetch = (pdl && co_resident && c->last_layer != layer && c->last_layer >= 0) ? 1 : 0;
     const float scale_log2 = c->scale * 1.4426950408889634f;
 
     cudaLaunchConfig_t lc;
