@@ -98,6 +98,9 @@ bool derive(const lar_config_t* c, Derived& d) {
     // number of CTAs (none is idle, merges stay k-way).  Whole units per CTA wherever that keeps the busiest
     // CTA within 25 % of the average (nothing to merge across CTAs); equal tile ranges otherwise.
     d.ctas = c->decode_ctas ? c->decode_ctas : kDefaultDecodeCtas;
+    // 128-byte rows in many short units: the per-unit work of a CTA (queries in, partials merged, row out) weighs
+    // more than its streaming; two CTAs per SM share it
+    if (!c->decode_ctas && c->head_dim == 64 && d.units >= 2 * kDefaultDecodeCtas) d.ctas = 2 * kDefaultDecodeCtas;
     if (!c->decode_ctas && d.units < d.ctas) d.ctas = d.units * (d.ctas / d.units);
     {
         const long long per = ((long long)d.units + d.ctas - 1) / d.ctas;
@@ -149,24 +152,16 @@ void make_layout(const lar_config_t* c, const Derived& d, Layout& L) {
 
 
 // Launch shape of the decode kernel.
-// bf16: persistent streaming kernel, one CTA per SM, W consumer warps and a ring of NS 16-row K/V stages;
-// a CTA stays below half of the SM's shared memory so that the next layer's kernel can move in and fill
-// its ring while this one is still streaming (programmatic dependent launch).
+// bf16: persistent streaming kernel, one CTA per SM, W consumer warps and a ring of NS 32-row K/V stages.  Measured on
+// B200: four consumers with two stages each stream as fast as anything deeper; letting a second CTA per SM in (so that
+// the next layer's kernel could fill its ring early) buys less than the stages it costs.
 // fp32: one cluster of X CTAs per unit, W warps per CTA, NS stages per warp.
 void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
     if (c->dtype == LAR_BF16) {
-        const int W = c->warps_per_cta ? c->warps_per_cta : 3;
-        int NS = c->stages;
-        if (NS == 0) {
-            const int budget = 113 * 1024;  // two CTAs (+ 1 KB each of system use) share the 228 KB of an SM
-            const int stage = 2 * (c->head_dim / 64) * lar::kStreamTile * 128 + 16;
-            const int fixed = c->head_dim == 64 ? lar::stream_fixed_smem_bytes(64, d.group, W) : lar::stream_fixed_smem_bytes(128, d.group, W);
-            NS = (budget - fixed) / stage;
-            if (NS > 32) NS = 32;
-        }
+        const int W = c->warps_per_cta ? c->warps_per_cta : 4;
+        int NS = c->stages ? c->stages : 2 * W;
         // a stage must always be read by the same consumer warp: ring depth = a multiple of W
         NS = NS / W * W;
-        if (c->stages == 0 && NS < 2 * W) NS = 2 * W;  // rather a deep ring than two CTAs per SM
         if (NS < W) NS = W;
         if (NS < 2) NS = 2;
         p.kv_splits = 1;
