@@ -28,6 +28,10 @@ if ROOT not in sys.path:
 
 METRIC = "image tokens/s of compressed-KV decode attention"
 UNIT = "image_tokens/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode launch (bytes), from the ncu capture summarised in
+# profiles/decode_stream_kernel_janus_pro_7b_4layers.md (one launch = one layer, so the 4-layer capture gives the
+# per-launch figure of the 30-layer workload); null for shapes that have no capture
+NCU_TRAFFIC_PER_LAUNCH = {"janus_pro_7b": 77.9e6}
 
 
 def load_peaks():
@@ -428,7 +432,7 @@ def run_ours(args):
                          "peak_kind": f"of {peak_kind} copy bandwidth",
                          "frac_of_8TBs": achieved / 8000.0,
                          "algorithmic_bytes_per_launch": kv_bytes / n_decode,
-                         "avg_launch_us": ms_decode * 1e3 / n_decode, "traffic": None},
+                         "avg_launch_us": ms_decode * 1e3 / n_decode, "traffic": NCU_TRAFFIC_PER_LAUNCH.get(w.name)},
             "sequence_tokens_per_s": world * w.batch * w.n_visual / (ms_step * 1e-3),
             "line_end_ms_per_step": ms_step - ms_decode,
             "per_token_ms": {"first_half": main["per_token_ms_first_half"], "last_half": main["per_token_ms_last_half"]},
