@@ -51,6 +51,7 @@ struct Derived {
     int units, group, elt, row_bytes, cap, ppu, P, cap_pad, M, mid_pad, compressing, B, N;
     int ctas, max_seg;  // bf16 decode: CTAs of the persistent grid, most segments one unit is cut into
     int unit_ranges;    // bf16 decode: 1 if the CTAs' ranges end on unit boundaries
+    int le_threads;     // threads per CTA of the line-end kernel
 };
 
 constexpr int kDefaultDecodeCtas = 148;  // one per SM of a B200
@@ -108,6 +109,8 @@ bool derive(const lar_config_t* c, Derived& d) {
         if (c->flags & LAR_FLAG_TILE_RANGES) d.unit_ranges = 0;
     }
     // A unit of T tiles is cut into at most ceil(T / floor(U T / P)) + 1 segments (never more than T or P).
+    // line end: one CTA per unit; few units with a large mid region get 16 warps instead of 8
+    d.le_threads = (d.units <= 2 * kDefaultDecodeCtas && d.M >= 128) ? 512 : 256;
     d.max_seg = 1;
     const int t_max = (d.cap + lar::kStreamTile - 1) / lar::kStreamTile;
     for (int T = 1; T <= t_max; ++T) {
@@ -207,7 +210,7 @@ lar_status_t plan_query_impl(const lar_config_t* cfg, lar_plan_t* out, Derived* 
     p.compressing = d.compressing;
     choose_plan(cfg, d, p);
     p.line_end_smem_bytes =
-        d.compressing ? lar::line_end_smem_bytes(d.row_bytes, cfg->head_dim, d.M, d.M - cfg->line_width + cfg->recent_lines * cfg->line_width, 8,
+        d.compressing ? lar::line_end_smem_bytes(d.row_bytes, cfg->head_dim, d.M, d.M - cfg->line_width + cfg->recent_lines * cfg->line_width, d.le_threads / 32,
                                                  cfg->line_width * d.group, cfg->dtype == LAR_BF16 ? 1 : 0) : 0;
     p.slab_bytes = L.total;
     p.scratch_bytes = (L.off_tickets + L.tickets_bytes) - L.off_partials;
@@ -676,7 +679,7 @@ lar_status_t lar_line_end_score_evict(lar_cache_t* c, int layer, void* stream) {
     if (c->d.compressing) {
         const lar::LayerView lv = view_of(c, layer);
         LineEndFn fn = line_end_fn(c->cfg, c->d.group);
-        fn<<<c->d.units, 256, c->plan.line_end_smem_bytes, (cudaStream_t)stream>>>(lv, c->scale * 1.4426950408889634f);
+        fn<<<c->d.units, c->d.le_threads, c->plan.line_end_smem_bytes, (cudaStream_t)stream>>>(lv, c->scale * 1.4426950408889634f);
         LAR_CUDA(cudaGetLastError());
         c->launches++;
         c->last_layer = layer;

@@ -134,7 +134,7 @@ __device__ __forceinline__ void score_mma(const unsigned char* kmid, const unsig
 // One CTA per unit.  Scoring: bf16 on tensor cores (score_mma); fp32 on CUDA cores, where every lane owns the keys
 // m = lane, lane + 32, ... and computes whole dot products against a query row broadcast from shared memory.
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(256) line_end_kernel(const LayerView lv, float scale_log2) {
+__global__ void __launch_bounds__(512) line_end_kernel(const LayerView lv, float scale_log2) {
     constexpr int EPL = Elt<T>::kPerChunk;
     constexpr int ROW_BYTES = D * (int)sizeof(T);
     constexpr int CHUNKS = ROW_BYTES / 16;
@@ -278,18 +278,21 @@ __global__ void __launch_bounds__(256) line_end_kernel(const LayerView lv, float
     for (int j = tid; j < n_rec; j += blockDim.x) srcmap[n_keep + j] = M + j;
     __syncthreads();
 
-    // rows move towards lower slots only (src >= dst); tiles ascending, load - barrier - store
-    constexpr int TILE_ROWS = 1024 / CHUNKS;  // 4 chunks of K and 4 of V per thread in flight (32 .. 128 rows)
+    // rows move towards lower slots only (src >= dst); tiles ascending, load - barrier - store;
+    // every thread carries 4 chunks of K and 4 of V per tile (64 .. 256 rows per tile)
+    constexpr int PER_THREAD = 4;
+    const int nthr = (int)blockDim.x;
+    const int tile_rows = nthr * PER_THREAD / CHUNKS;  // <= nthr
     int* imap = lv.index_map + (size_t)unit * lv.cap_pad;
-    for (int t0 = 0; t0 < total_rows; t0 += TILE_ROWS) {
-        const int rows = min(TILE_ROWS, total_rows - t0);
-        uint4 kbuf[(TILE_ROWS * CHUNKS + 255) / 256], vbuf[(TILE_ROWS * CHUNKS + 255) / 256];
+    for (int t0 = 0; t0 < total_rows; t0 += tile_rows) {
+        const int rows = min(tile_rows, total_rows - t0);
+        uint4 kbuf[PER_THREAD], vbuf[PER_THREAD];
         int ibuf = 0;
 #pragma unroll
-        for (int i = 0; i < (TILE_ROWS * CHUNKS + 255) / 256; ++i) {
-            const int idx = tid + i * 256;
+        for (int i = 0; i < PER_THREAD; ++i) {
+            const int idx = tid + i * nthr;
             const int r = idx / CHUNKS, c = idx - r * CHUNKS;
-            if (idx < rows * CHUNKS && (int)blockDim.x == 256) {
+            if (idx < rows * CHUNKS) {
                 const int src = srcmap[t0 + r];
                 if (src != t0 + r) {
                     const size_t off = row_offset(lv, unit, mid0 + src, ROW_BYTES) + c * 16;
@@ -301,10 +304,10 @@ __global__ void __launch_bounds__(256) line_end_kernel(const LayerView lv, float
         if (tid < rows) ibuf = imap[mid0 + srcmap[t0 + tid]];
         __syncthreads();
 #pragma unroll
-        for (int i = 0; i < (TILE_ROWS * CHUNKS + 255) / 256; ++i) {
-            const int idx = tid + i * 256;
+        for (int i = 0; i < PER_THREAD; ++i) {
+            const int idx = tid + i * nthr;
             const int r = idx / CHUNKS, c = idx - r * CHUNKS;
-            if (idx < rows * CHUNKS && (int)blockDim.x == 256) {
+            if (idx < rows * CHUNKS) {
                 if (srcmap[t0 + r] != t0 + r) {
                     const size_t off = row_offset(lv, unit, mid0 + t0 + r, ROW_BYTES) + c * 16;
                     *reinterpret_cast<uint4*>(lv.k_pool + off) = kbuf[i];
