@@ -125,7 +125,8 @@ struct Elt<float> {
 
 // byte address of row `slot` of a unit inside a pool
 __device__ __forceinline__ size_t row_offset(const LayerView& lv, int unit, int slot, int row_bytes) {
-    const int page = lv.page_table[unit * lv.pages_per_unit + slot / lv.page_tokens];
+    const int pidx = unit * lv.pages_per_unit + slot / lv.page_tokens;
+    const int page = lv.identity_pages ? pidx : lv.page_table[pidx];
     return (static_cast<size_t>(page) * lv.page_tokens + (slot % lv.page_tokens)) * row_bytes;
 }
 

@@ -109,8 +109,12 @@ bool derive(const lar_config_t* c, Derived& d) {
         if (c->flags & LAR_FLAG_TILE_RANGES) d.unit_ranges = 0;
     }
     // A unit of T tiles is cut into at most ceil(T / floor(U T / P)) + 1 segments (never more than T or P).
-    // line end: one CTA per unit; few units with a large mid region get 16 warps instead of 8
-    d.le_threads = (d.units <= 2 * kDefaultDecodeCtas && d.M >= 128) ? 512 : 256;
+    // line end: one CTA per unit, 8 warps; few units with a large mid region get one warp per 16 guide rows (16..32 warps)
+    d.le_threads = 256;
+    if (d.units <= 2 * kDefaultDecodeCtas && d.M >= 128) {
+        const int blocks = (c->line_width * d.group + 15) / 16;
+        d.le_threads = 32 * (blocks < 16 ? 16 : blocks > 32 ? 32 : blocks);
+    }
     d.max_seg = 1;
     const int t_max = (d.cap + lar::kStreamTile - 1) / lar::kStreamTile;
     for (int T = 1; T <= t_max; ++T) {

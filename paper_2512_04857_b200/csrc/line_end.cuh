@@ -134,7 +134,7 @@ __device__ __forceinline__ void score_mma(const unsigned char* kmid, const unsig
 // One CTA per unit.  Scoring: bf16 on tensor cores (score_mma); fp32 on CUDA cores, where every lane owns the keys
 // m = lane, lane + 32, ... and computes whole dot products against a query row broadcast from shared memory.
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(512) line_end_kernel(const LayerView lv, float scale_log2) {
+__global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv, float scale_log2) {
     constexpr int EPL = Elt<T>::kPerChunk;
     constexpr int ROW_BYTES = D * (int)sizeof(T);
     constexpr int CHUNKS = ROW_BYTES / 16;
