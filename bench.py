@@ -34,6 +34,20 @@ UNIT = "image_tokens/s"
 NCU_TRAFFIC_PER_LAUNCH = {"janus_pro_7b": 77.9e6}
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_value(images_per_rank, n_visual, world, ms_per_step_max):
+    """Image tokens/s of all ranks together: every rank is a replica doing the same work (weak scaling)."""
+    return world * images_per_rank * n_visual / (ms_per_step_max * 1e-3)
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -404,11 +418,8 @@ def run_ours(args):
         return res
 
     main = bench_workload(w, args.steps, args.warmup, True)
-    ms = torch.tensor([main["ms_per_step"], main["decode_ms_per_step"]], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    ms_step, ms_decode = float(ms[0]), float(ms[1])
-    value = world * w.images * w.n_visual / (ms_step * 1e-3)
+    ms_step, ms_decode = max_over_ranks([main["ms_per_step"], main["decode_ms_per_step"]], dist, dev)
+    value = whole_job_value(w.images, w.n_visual, world, ms_step)
     kv_bytes = w.kv_bytes_per_generation()
     n_decode = w.n_visual * w.n_layers
     achieved = kv_bytes / (ms_decode * 1e-3) / 1e9
