@@ -8,7 +8,7 @@ paper_2512_04857_b200.workloads) and resident in HBM before the timed region; th
 sequences are captured once into CUDA graphs and replayed.  All layers are cycled every token, so
 the working set (GBs) is far larger than L2.
 
-Prints ONE JSON line (see README for the keys).  `--impl reference` times the CPU oracle
+Prints ONE JSON line.  `--impl reference` times the CPU oracle
 on a bounded sample instead.
 """
 from __future__ import annotations
@@ -28,9 +28,9 @@ if ROOT not in sys.path:
 
 METRIC = "image tokens/s of compressed-KV decode attention"
 UNIT = "image_tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode launch (bytes), from the ncu capture summarised in
-# profiles/decode_stream_kernel_janus_pro_7b_4layers.md (one launch = one layer, so the 4-layer capture gives the
-# per-launch figure of the 30-layer workload); null for shapes that have no capture
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode launch (bytes), from an ncu capture of a 4-layer case of
+# the same shape and launch configuration (one launch = one layer, so the capture gives the per-launch figure of the
+# full workload); null for shapes that have no capture
 NCU_TRAFFIC_PER_LAUNCH = {"janus_pro_7b": 77.9e6}
 
 
