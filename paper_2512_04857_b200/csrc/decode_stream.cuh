@@ -15,8 +15,7 @@
 //
 // Inside a CTA three roles run concurrently, coupled only by mbarriers (every wait is bounded):
 //   warp 0           producer: walks the CTA's tile range and keeps a ring of NS stages filled with
-//                    K and V tiles (cp.async.bulk.tensor, 2-D tiled, 128-byte swizzle); also fetches
-//                    the queries (and the step's new k, v row) of each segment into a small ring.
+//                    K and V tiles (cp.async.bulk.tensor, 3-D tiled, 128-byte swizzle).
 //   warps 1 .. W     consumers: tile j of the range goes to consumer j % W:
 //                        S = Q K^T     mma.sync m16n8k16 (bf16 in, fp32 out), rows = the G heads
 //                        online softmax in fp32 (base-2, scale folded into the logits)
@@ -24,7 +23,8 @@
 //                                      layout is the B-operand layout of P^T, V^T fragments come from
 //                                      ldmatrix.trans, and no accumulator row is wasted on padding
 //                    and at the end of a segment each consumer leaves its partial in shared memory.
-//   warp W + 1       epilogue: merges the W partials of a segment with the step's own token,
+//   warp W + 1       epilogue: fetches the queries (and the step's new k, v row) of each segment into a
+//                    small ring; merges the W partials of a segment with the step's own token,
 //                    writes the output row (or the scratch partial + ticket), stores the new K/V
 //                    row, the index-map entry and the guide-queue row.
 // The producer never waits for arithmetic, so the HBM stream is continuous across unit boundaries.
@@ -256,11 +256,29 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
     const int u0 = (int)(t_begin / T);
     const int n_segs = n_tiles > 0 ? (int)((t_end - 1) / T) - u0 + 1 : 0;
 
+    // One lane requests the inputs of segment `seg`: its queries and, where the segment closes its unit in a fused
+    // step, the new k and v rows.  Issued by the epilogue warp, which is idle when a launch starts, so that the
+    // producer's first K/V copies are not queued behind them.
+    auto issue_inputs = [&](int seg) -> bool {
+        const int slot = seg % NQ;
+        if (seg >= NQ && !LAR_WAIT(17, true, wait_or_abort(bar_qempty + slot * 8, (uint32_t)((seg / NQ - 1) & 1), abort_flag))) return false;
+        const int unit = u0 + seg;
+        const bool closes = (long long)(unit + 1) * T <= t_end;  // the segment holds the unit's last tile
+        const bool with_kv = a.fused && closes;
+        const uint32_t bar = bar_qfull + slot * 8, dst = qring + slot * QENT;
+        mbar_expect_tx(bar, (uint32_t)((G + (with_kv ? 2 : 0)) * D * 2));
+        bulk_g2s(dst, reinterpret_cast<const T16*>(a.q) + (size_t)unit * G * D, G * D * 2, bar);
+        if (with_kv) {
+            bulk_g2s(dst + G * D * 2, reinterpret_cast<const T16*>(a.k_new) + (size_t)unit * D, D * 2, bar);
+            bulk_g2s(dst + (G + 1) * D * 2, reinterpret_cast<const T16*>(a.v_new) + (size_t)unit * D, D * 2, bar);
+        }
+        return true;
+    };
+
     if (warp == 0) {
         // =========================================================================== producer
         bool dep_waited = !a.prefetch;
         bool ok = true;
-        int q_next = 0;  // next segment whose inputs have not been requested yet (lane 0)
         const int fill_end = n_tiles < NS ? n_tiles : NS;
 
         auto describe = [&](int jj, int& y, int& rows, int& tile) {
@@ -277,22 +295,6 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
                 y = 0;
             }
         };
-        auto issue_inputs = [&](int seg) -> bool {  // lane 0: q (and the step's k, v) of segment `seg`
-            const int slot = seg % NQ;
-            if (seg >= NQ && !LAR_WAIT(17, true, wait_or_abort(bar_qempty + slot * 8, (uint32_t)((seg / NQ - 1) & 1), abort_flag))) return false;
-            const int unit = u0 + seg;
-            const bool closes = (long long)(unit + 1) * T <= t_end;  // the segment holds the unit's last tile
-            const bool with_kv = a.fused && closes;
-            const uint32_t bar = bar_qfull + slot * 8, dst = qring + slot * QENT;
-            mbar_expect_tx(bar, (uint32_t)((G + (with_kv ? 2 : 0)) * D * 2));
-            bulk_g2s(dst, reinterpret_cast<const T16*>(a.q) + (size_t)unit * G * D, G * D * 2, bar);
-            if (with_kv) {
-                bulk_g2s(dst + G * D * 2, reinterpret_cast<const T16*>(a.k_new) + (size_t)unit * D, D * 2, bar);
-                bulk_g2s(dst + (G + 1) * D * 2, reinterpret_cast<const T16*>(a.v_new) + (size_t)unit * D, D * 2, bar);
-            }
-            return true;
-        };
-
         // Lane 0 issues; all lanes look the page ids of a batch of 32 tiles up together, one batch ahead.
         // Stage and phase advance incrementally (no division in the per-tile path).  A fresh mbarrier lets a
         // wait on parity 1 pass, so the first trip round the ring does not wait for the consumers.
@@ -320,11 +322,6 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
                 const int yi = __shfl_sync(0xffffffffu, y, i), rti = __shfl_sync(0xffffffffu, rt, i);
                 if (lane == 0 && ok) {
                     const int ri = rti & 0xff;
-                    if (dep_waited && (j == 0 || (rti >> 8) == 0)) {
-                        // first tile of a segment: its inputs and those of the next segment must be on their way
-                        const int seg_now = (int)((t_begin + j) / T) - u0;
-                        while (ok && q_next < n_segs && q_next <= seg_now + 1) ok = issue_inputs(q_next++);
-                    }
                     if (ok) ok = LAR_WAIT(16, true, wait_or_abort(bar_empty + stage * 8, empty_parity, abort_flag));
                     if (ok) {
                         const uint32_t bar = bar_full + stage * 8, dst = ring + (uint32_t)stage * TR::STAGE_BYTES;
@@ -348,10 +345,6 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
                     grid_dep_launch();
                     LAR_STAMP(2);
                     dep_waited = true;
-                    if (lane == 0) {
-                        const int seg_now = (int)((t_begin + j) / T) - u0;
-                        while (ok && q_next < n_segs && q_next <= seg_now + 1) ok = issue_inputs(q_next++);
-                    }
                 }
             }
         }
@@ -523,6 +516,9 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
         grid_dep_wait();
         grid_dep_launch();
         bool ok = true;
+        if (lane == 0)
+            for (int sg = 0; sg < NQ && sg < n_segs && ok; ++sg) ok = issue_inputs(sg);  // the input ring's first round
+        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
         T16* outp = reinterpret_cast<T16*>(a.out);
         // What closing a unit needs from global memory (the page that takes the new row, the unit's length
         // in device memory) is requested one segment ahead, so that its latency never stalls this warp.
@@ -651,6 +647,9 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_pempty + buf * 8);
             LAR_STAMP(10);
+            // this segment's slot of the input ring is free once every consumer has taken its fragments: refill it
+            if (lane == 0 && seg + NQ < n_segs) ok = issue_inputs(seg + NQ);
+            if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
 
             if (opens && closes) {
                 // the whole unit lies in this CTA
