@@ -496,6 +496,28 @@ def run_ours(args):
                 pt["full_cache_ms_per_step"] = rf["ms_per_step"]
                 pt["speedup_vs_full_cache"] = rf["ms_per_step"] / rc["ms_per_step"]
             line["batch_sweep"]["points"].append(pt)
+    # ---- budget-ratio sweep at a given batch (the layout of the paper's efficiency table; not the headline line)
+    if args.ratio_sweep:
+        wr = W.WORKLOADS[args.sweep_workload]
+        if args.sweep_images:
+            wr = wr.scaled(batch=2 * args.sweep_images, images=args.sweep_images)
+        rf = bench_workload(wr.full_cache(), 1, 1, False, input_lines=2)
+        full_slab = lar.lar_cache_slab_bytes(lar.config_from_workload(wr.full_cache()))
+        line["ratio_sweep"] = {"workload": wr.name, "images": wr.images, "sequences": wr.batch,
+                               "full_cache": {"ms_per_step": rf["ms_per_step"], "kv_slab_gb": full_slab / 1e9,
+                                              "value": world * wr.images * wr.n_visual / (rf["ms_per_step"] * 1e-3)},
+                               "points": []}
+        for b in [int(x) for x in args.ratio_sweep.split(",")]:
+            w2 = wr.scaled(budget_lines=b, recent_lines=max(1, (b - 2) // 2), anchor_len=wr.line_width)
+            rc = bench_workload(w2, 1, 1, False, input_lines=2)
+            slab = lar.lar_cache_slab_bytes(lar.config_from_workload(w2))
+            ach = w2.kv_bytes_per_generation() / (rc["decode_ms_per_step"] * 1e-3) / 1e9
+            line["ratio_sweep"]["points"].append(
+                {"budget_lines": b, "budget_tokens": w2.budget_tokens, "ratio": f"{b}/{w2.n_lines}",
+                 "recent_lines": w2.recent_lines, "mid_len": w2.mid_len,
+                 "value": world * w2.images * w2.n_visual / (rc["ms_per_step"] * 1e-3), "ms_per_step": rc["ms_per_step"],
+                 "speedup_vs_full_cache": rf["ms_per_step"] / rc["ms_per_step"], "kv_slab_gb": slab / 1e9,
+                 "memory_saving": 1.0 - slab / full_slab, "roofline_achieved_gbs": ach, "roofline_frac": ach / peak})
     # ---- CPU oracle on the host cores (rank 0, N = 1 only)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = {k: v for k, v in cpu_baseline(w).items() if k not in ("seconds", "units")}
@@ -516,6 +538,8 @@ def main():
     ap.add_argument("--also", default="", help="comma-separated extra workloads reported under 'also'")
     ap.add_argument("--batch-sweep", default="", help="comma-separated image counts: sweep the batch of --sweep-workload")
     ap.add_argument("--sweep-workload", default="gqa_1024")
+    ap.add_argument("--ratio-sweep", default="", help="comma-separated line budgets: sweep the budget of --sweep-workload")
+    ap.add_argument("--sweep-images", type=int, default=0, help="images per batch in --ratio-sweep (0: the workload's own)")
     ap.add_argument("--kv-splits", type=int, default=0)
     ap.add_argument("--warps", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
