@@ -12,6 +12,18 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
 
 
+def pytest_sessionstart(session):
+    """The tests call the CUDA library through its C ABI: compile it (and the C oracle) if a fresh checkout has no
+    binaries yet.  nvcc cross-compiles for sm_100a without a GPU."""
+    try:
+        from paper_2512_04857_b200 import build as lib_build
+        from oracle import build as oracle_build
+        lib_build.build()
+        oracle_build.build()
+    except Exception as e:          # the tests that need the library will say so themselves
+        print(f"[conftest] build skipped: {e}")
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch
