@@ -28,8 +28,10 @@
 //                    writes the output row (or the scratch partial + ticket), stores the new K/V
 //                    row, the index-map entry and the guide-queue row.
 // The producer never waits for arithmetic, so the HBM stream is continuous across unit boundaries.
-// With programmatic dependent launch the producer fills its ring with tiles of this layer's cache
-// while the preceding kernel (another layer) is still running; everything else waits for it.
+// Launched with programmatic dependent launch, the CTAs of the next layer's kernel move in as SMs free up
+// and wait for the preceding kernel in griddepcontrol.wait; where the host asks for it (prefetch = 1: two
+// CTAs fit per SM) the producer first fills its ring with tiles of this layer's cache, which the preceding
+// kernel (another layer) does not touch.
 #pragma once
 #include <cuda.h>
 
