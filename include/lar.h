@@ -87,7 +87,7 @@ typedef struct lar_config {
     int32_t warps_per_cta; /* decode warps: bf16 consumer warps per CTA, 0 auto, else 1..6;
                               fp32 warps per CTA, 0 auto, else 1..8 */
     int32_t stages;        /* 16-row K/V stages: bf16 depth of the CTA's ring, 0 auto, else 2..32 (rounded
-                              down to a multiple of the consumer warps, at least one per warp);
+                              down to a common multiple of the consumer warps and the two producer warps);
                               fp32 stages in flight per warp, 0 auto, else 1..4 */
     uint32_t page_seed;    /* seed of LAR_FLAG_SHUFFLE_PAGES */
     int32_t decode_ctas;   /* bf16 only: CTAs of the persistent decode grid: 0 selects 148 (one per SM), else 1..1024 */

@@ -14,16 +14,16 @@
 // unit checks it against the unit's length in device memory before advancing that.
 //
 // Inside a CTA three roles run concurrently, coupled only by mbarriers (every wait is bounded):
-//   warp 0           producer: walks the CTA's tile range and keeps a ring of NS stages filled with
-//                    K and V tiles (cp.async.bulk.tensor, 3-D tiled, 128-byte swizzle).
-//   warps 1 .. W     consumers: tile j of the range goes to consumer j % W:
+//   warps 0, 1       producers: walk the CTA's tile range (every other tile each) and keep a ring of NS
+//                    stages filled with K and V tiles (cp.async.bulk.tensor, 3-D tiled, 128-byte swizzle).
+//   next W warps     consumers: tile j of the range goes to consumer j % W:
 //                        S = Q K^T     mma.sync m16n8k16 (bf16 in, fp32 out), rows = the G heads
 //                        online softmax in fp32 (base-2, scale folded into the logits)
 //                        O^T += V^T P^T  same instruction with the d rows as M: the logits' accumulator
 //                                      layout is the B-operand layout of P^T, V^T fragments come from
 //                                      ldmatrix.trans, and no accumulator row is wasted on padding
 //                    and at the end of a segment each consumer leaves its partial in shared memory.
-//   warp W + 1       epilogue: fetches the queries (and the step's new k, v row) of each segment into a
+//   last warp        epilogue: fetches the queries (and the step's new k, v row) of each segment into a
 //                    small ring; merges the W partials of a segment with the step's own token,
 //                    writes the output row (or the scratch partial + ticket), stores the new K/V
 //                    row, the index-map entry and the guide-queue row.
@@ -119,6 +119,7 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {
 
 // ---- shared-memory plan of decode_stream_kernel (host and device agree through these) -------------
 constexpr int kMaxConsumers = 6;  // consumer warps per CTA at most
+constexpr int kProducers = 2;     // producer warps per CTA: tile j is fetched by producer j % kProducers
 __host__ __device__ constexpr int stream_q_slots(int G) { return G <= 2 ? 8 : 4; }
 __host__ __device__ constexpr int stream_partial_bufs(int) { return 2; }  // partial buffers per CTA
 __host__ __device__ constexpr int stream_q_entry_bytes(int D, int G) { return ((G + 2) * D * 2 + 127) / 128 * 128; }
@@ -185,7 +186,7 @@ __device__ __forceinline__ int range_owner(long long t, long long total, int P) 
 }
 
 template <int D, int G>
-__global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs a, const __grid_constant__ TensorMaps tm) {
+__global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs a, const __grid_constant__ TensorMaps tm) {
     using TR = MmaTraits<D>;
     using T16 = __nv_bfloat16;
     constexpr int NQ = stream_q_slots(G);
@@ -196,7 +197,7 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
     extern __shared__ unsigned char smem_raw[];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int W = (int)(blockDim.x >> 5) - 2;  // consumer warps
+    const int W = (int)(blockDim.x >> 5) - kProducers - 1;  // consumer warps
     const int NS = a.n_stages;
     const int P = (int)gridDim.x, p = (int)blockIdx.x;
     const LayerView& lv = a.lv;
@@ -277,11 +278,16 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
         return true;
     };
 
-    if (warp == 0) {
-        // =========================================================================== producer
+    if (warp < kProducers) {
+        // =========================================================================== producers
+        // Producer pw fetches the tiles pw, pw + kProducers, ... of the CTA's range (a single thread sustains only one
+        // tiled copy per ~140 cycles, two keep the ring ahead of the consumers).  NS is a multiple of kProducers, so
+        // a stage is always filled by the same producer.
+        const int pw = warp;
         bool dep_waited = !a.prefetch;
         bool ok = true;
         const int fill_end = n_tiles < NS ? n_tiles : NS;
+        const int n_local = n_tiles > pw ? (n_tiles - pw + kProducers - 1) / kProducers : 0;
 
         auto describe = [&](int jj, int& y, int& rows, int& tile) {
             const long long t = t_begin + jj;
@@ -303,28 +309,35 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
         int y_n = 0, rt_n = 0;  // rt = rows | tile << 8
         {
             int r = 0, t = 0;
-            if (lane < n_tiles) describe(lane, y_n, r, t);
+            if (lane < n_local) describe(kProducers * lane + pw, y_n, r, t);
             rt_n = r | (t << 8);
         }
-        LAR_STAMP(1);
         // every cached row is read once per step: let it leave L2 first
         const uint64_t pol_stream = l2_policy_evict_first();
-        int stage = 0;
+        LAR_STAMP(1);
+        int stage = pw;
         uint32_t empty_parity = 1;
-        for (int j0 = 0; j0 < n_tiles; j0 += 32) {
+        for (int i0 = 0; i0 < n_local; i0 += 32) {
             const int y = y_n, rt = rt_n;
-            if (j0 + 32 + lane < n_tiles) {  // next batch: hides the table reads
+            if (i0 + 32 + lane < n_local) {  // next batch: hides the table reads
                 int r = 0, t = 0;
-                describe(j0 + 32 + lane, y_n, r, t);
+                describe(kProducers * (i0 + 32 + lane) + pw, y_n, r, t);
                 rt_n = r | (t << 8);
             }
-            const int cnt = n_tiles - j0 < 32 ? n_tiles - j0 : 32;
+            const int cnt = n_local - i0 < 32 ? n_local - i0 : 32;
             for (int i = 0; i < cnt; ++i) {
-                const int j = j0 + i;
+                const int j = kProducers * (i0 + i) + pw;
+                if (!dep_waited && j >= fill_end) {
+                    // the ring is full of this layer's cache; everything else depends on the preceding kernel
+                    grid_dep_wait();
+                    grid_dep_launch();
+                    LAR_STAMP(2);
+                    dep_waited = true;
+                }
                 const int yi = __shfl_sync(0xffffffffu, y, i), rti = __shfl_sync(0xffffffffu, rt, i);
                 if (lane == 0 && ok) {
                     const int ri = rti & 0xff;
-                    if (ok) ok = LAR_WAIT(16, true, wait_or_abort(bar_empty + stage * 8, empty_parity, abort_flag));
+                    ok = LAR_WAIT(16, true, wait_or_abort(bar_empty + stage * 8, empty_parity, abort_flag));
                     if (ok) {
                         const uint32_t bar = bar_full + stage * 8, dst = ring + (uint32_t)stage * TR::STAGE_BYTES;
                         if (ri > 0) {
@@ -336,17 +349,11 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
                             mbar_arrive(bar);  // nothing to fetch: release the consumer
                         }
                     }
-                    if (++stage == NS) {
-                        stage = 0;
+                    stage += kProducers;
+                    if (stage >= NS) {
+                        stage -= NS;
                         empty_parity ^= 1u;
                     }
-                }
-                if (!dep_waited && j == fill_end - 1) {
-                    // the ring is full of this layer's cache; everything else depends on the preceding kernel
-                    grid_dep_wait();
-                    grid_dep_launch();
-                    LAR_STAMP(2);
-                    dep_waited = true;
                 }
             }
         }
@@ -356,11 +363,11 @@ __global__ void __launch_bounds__(256, 2) decode_stream_kernel(const StreamArgs 
         }
         LAR_STAMP(3);
         if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
-    } else if (warp <= W) {
+    } else if (warp < kProducers + W) {
         // =========================================================================== consumers
         grid_dep_wait();
         grid_dep_launch();
-        const int cw = warp - 1;
+        const int cw = warp - kProducers;
         const int quad = lane & 3, qrow = lane >> 2;  // fragment coordinates
         bool ok = true;
         // This consumer takes tiles cw, cw + W, ... of the CTA's range.  NS is a multiple of W, so a stage is

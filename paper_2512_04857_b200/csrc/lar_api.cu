@@ -167,10 +167,11 @@ void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
     if (c->dtype == LAR_BF16) {
         const int W = c->warps_per_cta ? c->warps_per_cta : 4;
         int NS = c->stages ? c->stages : 2 * W;
-        // a stage must always be read by the same consumer warp: ring depth = a multiple of W
-        NS = NS / W * W;
-        if (NS < W) NS = W;
-        if (NS < 2) NS = 2;
+        // a stage must always be read by the same consumer warp and filled by the same producer warp:
+        // ring depth = a multiple of W and of the number of producers
+        const int step = W % lar::kProducers == 0 ? W : W * lar::kProducers;
+        NS = NS / step * step;
+        if (NS < step) NS = step;
         p.kv_splits = 1;
         p.warps_per_cta = W;
         p.stages = NS;
@@ -432,7 +433,7 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
         a.max_seg = c->d.max_seg;
         a.pool_row_base = layer * c->rows_per_layer;
         lc.gridDim = dim3((unsigned)c->d.ctas, 1, 1);
-        lc.blockDim = dim3((unsigned)(32 * (c->plan.warps_per_cta + 2)), 1, 1);
+        lc.blockDim = dim3((unsigned)(32 * (c->plan.warps_per_cta + lar::kProducers + 1)), 1, 1);
         lc.attrs = attrs;
         lc.numAttrs = na;
         DecodeStreamFn fn = decode_stream_fn(c->cfg, c->d.group);

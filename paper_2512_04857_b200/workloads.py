@@ -133,6 +133,14 @@ WORKLOADS: Dict[str, Workload] = {
     "lumina_768": _mk(name="lumina_768", n_layers=32, batch=8, images=4, n_q_heads=32, n_kv_heads=32,
                       head_dim=128, dtype="bf16", cond_len=128, line_width=49, n_lines=48, budget_lines=6,
                       anchor_len=49, recent_lines=2, seed=4, note="48 columns + 1 line-end token per row"),
+    # further shapes of the paper's tables (same generator; not the headline): LlamaGen-XXL (class-conditional, Table 2)
+    # and Janus-Pro-1B (Table 1, ablations)
+    "llamagen_xxl": _mk(name="llamagen_xxl", n_layers=48, batch=64, images=32, n_q_heads=24, n_kv_heads=24,
+                        head_dim=64, dtype="bf16", cond_len=1, line_width=24, n_lines=24, budget_lines=4,
+                        anchor_len=24, recent_lines=1, seed=6),
+    "janus_pro_1b": _mk(name="janus_pro_1b", n_layers=24, batch=32, images=16, n_q_heads=16, n_kv_heads=16,
+                        head_dim=128, dtype="bf16", cond_len=64, line_width=24, n_lines=24, budget_lines=4,
+                        anchor_len=24, recent_lines=1, seed=7, prefix_key_scale=1.5),
     "gqa_1024": _mk(name="gqa_1024", n_layers=32, batch=16, images=8, n_q_heads=32, n_kv_heads=8,
                     head_dim=128, dtype="bf16", cond_len=128, line_width=65, n_lines=64, budget_lines=8,
                     anchor_len=65, recent_lines=3, seed=5, note="64 columns + 1 line-end token per row"),

@@ -121,6 +121,6 @@ def test_full_cache_budget_and_overrides():
     p = lar.lar_plan_query(_cfg(dtype="fp32", kv_splits=4, warps_per_cta=8, stages=2, page_tokens=32))
     assert (p.kv_splits, p.warps_per_cta, p.stages, p.page_tokens) == (4, 8, 2, 32)
     p = lar.lar_plan_query(_cfg(warps_per_cta=3, stages=9, decode_ctas=40, page_tokens=64))
-    assert (p.warps_per_cta, p.stages, p.decode_ctas, p.page_tokens) == (3, 9, 40, 64)
+    assert (p.warps_per_cta, p.stages, p.decode_ctas, p.page_tokens) == (3, 6, 40, 64)   # ring depth: multiple of 3 consumers and 2 producers
     # 4 units of up to 2 tiles (36 slots, 32-row tiles) dealt to 40 CTAs: every tile may sit in a CTA of its own
     assert p.max_segments == 2
