@@ -59,7 +59,7 @@ struct StreamArgs {
     int len, n_tok;     // live rows per unit / visual tokens appended so far, before this step's append
     int unit_ranges;    // 1: CTA ranges end on unit boundaries
     int fused;          // 1: the step's token comes from k_new / v_new and is appended by this kernel
-    int prefetch;       // 1: cached K/V may be fetched before the preceding kernel has finished
+    int prefetch;       // > 0: that many tiles of cached K/V per CTA may be fetched before the preceding kernel has finished
     int n_units, n_stages, max_seg;
     int pool_row_base;  // first pool row of this layer in the tensor maps
 };
@@ -286,7 +286,8 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         const int pw = warp;
         bool dep_waited = !a.prefetch;
         bool ok = true;
-        const int fill_end = n_tiles < NS ? n_tiles : NS;
+        const int fill_cap = a.prefetch < NS ? a.prefetch : NS;
+        const int fill_end = n_tiles < fill_cap ? n_tiles : fill_cap;
         const int n_local = n_tiles > pw ? (n_tiles - pw + kProducers - 1) / kProducers : 0;
 
         auto describe = [&](int jj, int& y, int& rows, int& tile) {
@@ -328,7 +329,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             for (int i = 0; i < cnt; ++i) {
                 const int j = kProducers * (i0 + i) + pw;
                 if (!dep_waited && j >= fill_end) {
-                    // the ring is full of this layer's cache; everything else depends on the preceding kernel
+                    // the first tiles of this layer's cache are on their way; everything else depends on the preceding kernel
                     grid_dep_wait();
                     grid_dep_launch();
                     LAR_STAMP(2);

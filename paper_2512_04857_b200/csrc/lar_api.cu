@@ -386,10 +386,11 @@ lar_status_t launch_append(lar_cache* c, int layer, const void* k, const void* v
 lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k, const void* v, void* out, int fused,
                            cudaStream_t s) {
     const bool pdl = (c->cfg.flags & LAR_FLAG_PDL) != 0;
-    // Fetching cached K/V ahead of the dependency pays only if this launch's CTAs can move in beside the preceding
-    // kernel's (two per SM); otherwise they start when that kernel is done and want their inputs first.
-    const bool co_resident = c->cfg.dtype != LAR_BF16 || 2 * (c->plan.decode_smem_bytes + 1024) <= 228 * 1024;
-    const int prefetch = (pdl && co_resident && c->last_layer != layer && c->last_layer >= 0) ? 1 : 0;
+    // With programmatic dependent launch a CTA moves in as soon as an SM is free, a few microseconds before the
+    // preceding kernel is done.  It requests its first ring of cached K/V tiles then, so that arithmetic starts when
+    // the dependency resolves.
+    int prefetch = 0;
+    if (pdl && c->last_layer != layer && c->last_layer >= 0) prefetch = c->cfg.dtype == LAR_BF16 ? c->plan.stages : 1;
     const float scale_log2 = c->scale * 1.4426950408889634f;
 
     cudaLaunchConfig_t lc;
