@@ -100,8 +100,8 @@ bool derive(const lar_config_t* c, Derived& d) {
     // CTA within 25 % of the average (nothing to merge across CTAs); equal tile ranges otherwise.
     d.ctas = c->decode_ctas ? c->decode_ctas : kDefaultDecodeCtas;
     // 128-byte rows in many short units: the per-unit work of a CTA (queries in, partials merged, row out) weighs
-    // more than its streaming; two CTAs per SM share it
-    if (!c->decode_ctas && c->head_dim == 64 && d.units >= 2 * kDefaultDecodeCtas) d.ctas = 2 * kDefaultDecodeCtas;
+    // more than its streaming; three small CTAs per SM share it
+    if (!c->decode_ctas && c->head_dim == 64 && d.units >= 3 * kDefaultDecodeCtas) d.ctas = 3 * kDefaultDecodeCtas;
     if (!c->decode_ctas && d.units < d.ctas) d.ctas = d.units * (d.ctas / d.units);
     {
         const long long per = ((long long)d.units + d.ctas - 1) / d.ctas;
@@ -165,7 +165,8 @@ void make_layout(const lar_config_t* c, const Derived& d, Layout& L) {
 // fp32: one cluster of X CTAs per unit, W warps per CTA, NS stages per warp.
 void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
     if (c->dtype == LAR_BF16) {
-        const int W = c->warps_per_cta ? c->warps_per_cta : 4;
+        // (three CTAs per SM, chosen for 128-byte rows in many short units, get two consumers each)
+        const int W = c->warps_per_cta ? c->warps_per_cta : (d.ctas > 2 * kDefaultDecodeCtas && !c->decode_ctas ? 2 : 4);
         int NS = c->stages ? c->stages : 2 * W;
         // a stage must always be read by the same consumer warp and filled by the same producer warp:
         // ring depth = a multiple of W and of the number of producers
