@@ -102,6 +102,8 @@ bool derive(const lar_config_t* c, Derived& d) {
     // 128-byte rows in many short units: the per-unit work of a CTA (queries in, partials merged, row out) weighs
     // more than its streaming; three small CTAs per SM share it
     if (!c->decode_ctas && c->head_dim == 64 && d.units >= 3 * kDefaultDecodeCtas) d.ctas = 3 * kDefaultDecodeCtas;
+    // 256-byte rows: with three or more units per SM two CTAs per SM (two producers pairs, two epilogue warps) stream faster
+    if (!c->decode_ctas && c->head_dim == 128 && d.units >= 3 * kDefaultDecodeCtas) d.ctas = 2 * kDefaultDecodeCtas;
     if (!c->decode_ctas && d.units < d.ctas) d.ctas = d.units * (d.ctas / d.units);
     {
         const long long per = ((long long)d.units + d.ctas - 1) / d.ctas;
@@ -165,8 +167,9 @@ void make_layout(const lar_config_t* c, const Derived& d, Layout& L) {
 // fp32: one cluster of X CTAs per unit, W warps per CTA, NS stages per warp.
 void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
     if (c->dtype == LAR_BF16) {
-        // (three CTAs per SM, chosen for 128-byte rows in many short units, get two consumers each)
-        const int W = c->warps_per_cta ? c->warps_per_cta : (d.ctas > 2 * kDefaultDecodeCtas && !c->decode_ctas ? 2 : 4);
+        // (grids of two or three CTAs per SM get three or two consumers each)
+        const int per_sm = c->decode_ctas ? 1 : (d.ctas + kDefaultDecodeCtas - 1) / kDefaultDecodeCtas;  // CTAs per SM of the default grids
+        const int W = c->warps_per_cta ? c->warps_per_cta : (per_sm >= 3 ? 2 : per_sm == 2 ? 3 : 4);
         int NS = c->stages ? c->stages : 2 * W;
         // a stage must always be read by the same consumer warp and filled by the same producer warp:
         // ring depth = a multiple of W and of the number of producers
