@@ -169,7 +169,8 @@ void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
     if (c->dtype == LAR_BF16) {
         // (grids of two or three CTAs per SM get three or two consumers each)
         const int per_sm = c->decode_ctas ? 1 : (d.ctas + kDefaultDecodeCtas - 1) / kDefaultDecodeCtas;  // CTAs per SM of the default grids
-        const int W = c->warps_per_cta ? c->warps_per_cta : (per_sm >= 3 ? 2 : per_sm == 2 ? 3 : 4);
+        // ... and a CTA that holds (part of) one long unit gets a fifth
+        const int W = c->warps_per_cta ? c->warps_per_cta : (per_sm >= 3 ? 2 : per_sm == 2 ? 3 : (d.units <= d.ctas && !c->decode_ctas) ? 5 : 4);
         int NS = c->stages ? c->stages : 2 * W;
         // a stage must always be read by the same consumer warp and filled by the same producer warp:
         // ring depth = a multiple of W and of the number of producers
