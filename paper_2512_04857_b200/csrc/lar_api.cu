@@ -102,8 +102,11 @@ bool derive(const lar_config_t* c, Derived& d) {
     // 128-byte rows in many short units: the per-unit work of a CTA (queries in, partials merged, row out) weighs
     // more than its streaming; three small CTAs per SM share it
     if (!c->decode_ctas && c->head_dim == 64 && d.units >= 3 * kDefaultDecodeCtas) d.ctas = 3 * kDefaultDecodeCtas;
-    // 256-byte rows: with three or more units per SM two CTAs per SM (two producers pairs, two epilogue warps) stream faster
-    if (!c->decode_ctas && c->head_dim == 128 && d.units >= 3 * kDefaultDecodeCtas) d.ctas = 2 * kDefaultDecodeCtas;
+    // 256-byte rows: with three or more short units (up to 8 tiles) per SM, two CTAs per SM (two pairs of producers, two
+    // epilogue warps) stream faster; long units are better served by one CTA with more consumers
+    if (!c->decode_ctas && c->head_dim == 128 && d.units >= 3 * kDefaultDecodeCtas &&
+        (d.cap + lar::kStreamTile - 1) / lar::kStreamTile <= 8)
+        d.ctas = 2 * kDefaultDecodeCtas;
     if (!c->decode_ctas && d.units < d.ctas) d.ctas = d.units * (d.ctas / d.units);
     {
         const long long per = ((long long)d.units + d.ctas - 1) / d.ctas;
