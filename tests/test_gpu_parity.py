@@ -44,7 +44,7 @@ def test_launch_shapes(splits, warps, stages):
     _check(rep, w)
 
 
-@pytest.mark.parametrize("ctas,warps,stages", [(1, 1, 2), (3, 2, 3), (7, 4, 5), (40, 3, 12), (148, 4, 0), (296, 1, 16),
+@pytest.mark.parametrize("ctas,warps,stages", [(1, 1, 2), (3, 2, 3), (7, 4, 5), (40, 3, 12), (148, 4, 0), (296, 1, 16), (148, 5, 10), (74, 6, 12),
                                                (1024, 4, 2)])
 @pytest.mark.parametrize("fused", [True, False])
 def test_stream_launch_shapes_bf16(ctas, warps, stages, fused):
