@@ -63,7 +63,7 @@ typedef enum { LAR_BF16 = 0, LAR_FP32 = 1 } lar_dtype_t;
                                         caller kernel using PDL waits on its own dependency before it
                                         triggers its dependents. */
 #define LAR_FLAG_SHUFFLE_PAGES 0x4u  /* test hook: assign physical pages in a pseudo-random order */
-#define LAR_FLAG_TILE_RANGES 0x8u    /* bf16 decode: always deal 16-row tiles (not whole units) to the CTAs, even
+#define LAR_FLAG_TILE_RANGES 0x8u    /* bf16 decode: always deal 32-row tiles (not whole units) to the CTAs, even
                                         where whole units would balance well enough */
 
 typedef struct lar_config {
@@ -86,11 +86,12 @@ typedef struct lar_config {
     int32_t kv_splits;     /* fp32 only: CTAs (one thread-block cluster) per unit in decode: 0 auto, else 1,2,4,8 */
     int32_t warps_per_cta; /* decode warps: bf16 consumer warps per CTA, 0 auto, else 1..6;
                               fp32 warps per CTA, 0 auto, else 1..8 */
-    int32_t stages;        /* 16-row K/V stages: bf16 depth of the CTA's ring, 0 auto, else 2..32 (rounded
+    int32_t stages;        /* K/V stages: bf16 depth of the CTA's ring of 32-row tiles, 0 auto, else 2..32 (rounded
                               down to a common multiple of the consumer warps and the two producer warps);
-                              fp32 stages in flight per warp, 0 auto, else 1..4 */
+                              fp32 16-row stages in flight per warp, 0 auto, else 1..4 */
     uint32_t page_seed;    /* seed of LAR_FLAG_SHUFFLE_PAGES */
-    int32_t decode_ctas;   /* bf16 only: CTAs of the persistent decode grid: 0 selects 148 (one per SM), else 1..1024 */
+    int32_t decode_ctas;   /* bf16 only: CTAs of the persistent decode grid: 0 lets the library choose (one to three per
+                              SM of a B200, or a multiple of the unit count when there are fewer units than SMs), else 1..1024 */
 } lar_config_t;
 
 /* What lar_cache_create derived from a config (introspection; also usable without a GPU). */

@@ -3,7 +3,7 @@
 //
 // Work decomposition.  The live rows of every unit = (sequence, KV head) are cut into 32-row tiles;
 // all tiles of the layer form one list (unit-major) that is dealt out in contiguous ranges to the CTAs
-// of the grid (one CTA per SM).  Where whole units can be dealt out evenly enough the ranges end on unit
+// of the grid (one to three CTAs per SM).  Where whole units can be dealt out evenly enough the ranges end on unit
 // boundaries; otherwise they are equal in tiles, so that every SM streams the same number of bytes
 // whatever the number of units.  The part of a unit that falls into one CTA is a *segment*.  A unit
 // that lies inside one CTA is finished there; a unit cut by a range boundary leaves one partial

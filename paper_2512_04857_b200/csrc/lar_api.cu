@@ -164,9 +164,9 @@ void make_layout(const lar_config_t* c, const Derived& d, Layout& L) {
 
 
 // Launch shape of the decode kernel.
-// bf16: persistent streaming kernel, one CTA per SM, W consumer warps and a ring of NS 32-row K/V stages.  Measured on
-// B200: four consumers with two stages each stream as fast as anything deeper; letting a second CTA per SM in (so that
-// the next layer's kernel could fill its ring early) buys less than the stages it costs.
+// bf16: persistent streaming kernel; per CTA two producer warps, W consumer warps, an epilogue warp and a ring of NS
+// 32-row K/V stages.  Measured on B200: two stages per consumer stream as fast as anything deeper; the consumer count
+// follows the grid (derive(): one to three CTAs per SM).
 // fp32: one cluster of X CTAs per unit, W warps per CTA, NS stages per warp.
 void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
     if (c->dtype == LAR_BF16) {
