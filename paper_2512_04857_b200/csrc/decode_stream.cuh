@@ -180,9 +180,17 @@ __device__ __forceinline__ float exp2_or_zero(float m_part, float m_all) {
     return m_part == -INFINITY ? 0.f : exp2f(m_part - m_all);
 }
 
-// CTA that owns item t of a list of `total` items dealt to P <= total CTAs as ranges [p total / P, (p + 1) total / P)
-__device__ __forceinline__ int range_owner(long long t, long long total, int P) {
-    return (int)(((t + 1) * P - 1) / total);
+// A list of n items is dealt to P <= n CTAs in contiguous ranges, the first n % P of them one item longer.
+// (32-bit arithmetic throughout: the host rejects configurations with 2^30 tiles or more per layer.)
+__device__ __forceinline__ int range_begin(int n, int P, int p) {
+    const int q = n / P, r = n - q * P;
+    return p * q + (p < r ? p : r);
+}
+// CTA that owns item t
+__device__ __forceinline__ int range_owner(int t, int n, int P) {
+    const int q = n / P, r = n - q * P;
+    const int head = r * (q + 1);
+    return t < head ? t / (q + 1) : r + (t - head) / q;
 }
 
 template <int D, int G>
@@ -239,25 +247,25 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     // ---- the layer's tile list and this CTA's range of it
     const int len = a.len, n_tok = a.n_tok;
     const int T = len > 0 ? (len + kStreamTile - 1) / kStreamTile : 1;  // an empty cache is one tile of 0 rows
-    const long long total = (long long)a.n_units * T;
-    long long t_begin = 0, t_end = 0;
+    const int total = a.n_units * T;
+    int t_begin = 0, t_end = 0;
     int Pe;  // CTAs that get work: every range is non-empty
     if (a.unit_ranges) {
         Pe = a.n_units < P ? a.n_units : P;
         if (p < Pe) {
-            t_begin = ((long long)p * a.n_units / Pe) * T;
-            t_end = ((long long)(p + 1) * a.n_units / Pe) * T;
+            t_begin = range_begin(a.n_units, Pe, p) * T;
+            t_end = range_begin(a.n_units, Pe, p + 1) * T;
         }
     } else {
-        Pe = total < P ? (int)total : P;
+        Pe = total < P ? total : P;
         if (p < Pe) {
-            t_begin = (long long)p * total / Pe;
-            t_end = (long long)(p + 1) * total / Pe;
+            t_begin = range_begin(total, Pe, p);
+            t_end = range_begin(total, Pe, p + 1);
         }
     }
-    const int n_tiles = (int)(t_end - t_begin);
-    const int u0 = (int)(t_begin / T);
-    const int n_segs = n_tiles > 0 ? (int)((t_end - 1) / T) - u0 + 1 : 0;
+    const int n_tiles = t_end - t_begin;
+    const int u0 = t_begin / T;
+    const int n_segs = n_tiles > 0 ? (t_end - 1) / T - u0 + 1 : 0;
 
     // One lane requests the inputs of segment `seg`: its queries and, where the segment closes its unit in a fused
     // step, the new k and v rows.  Issued by the epilogue warp, which is idle when a launch starts, so that the
@@ -266,7 +274,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         const int slot = seg % NQ;
         if (seg >= NQ && !LAR_WAIT(17, true, wait_or_abort(bar_qempty + slot * 8, (uint32_t)((seg / NQ - 1) & 1), abort_flag))) return false;
         const int unit = u0 + seg;
-        const bool closes = (long long)(unit + 1) * T <= t_end;  // the segment holds the unit's last tile
+        const bool closes = (unit + 1) * T <= t_end;  // the segment holds the unit's last tile
         const bool with_kv = a.fused && closes;
         const uint32_t bar = bar_qfull + slot * 8, dst = qring + slot * QENT;
         mbar_expect_tx(bar, (uint32_t)((G + (with_kv ? 2 : 0)) * D * 2));
@@ -291,9 +299,9 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         const int n_local = n_tiles > pw ? (n_tiles - pw + kProducers - 1) / kProducers : 0;
 
         auto describe = [&](int jj, int& y, int& rows, int& tile) {
-            const long long t = t_begin + jj;
-            const int unit = (int)(t / T);
-            tile = (int)(t - (long long)unit * T);
+            const int t = t_begin + jj;
+            const int unit = t / T;
+            tile = t - unit * T;
             const int row0 = tile * kStreamTile;
             rows = len - row0 < kStreamTile ? len - row0 : kStreamTile;
             if (rows > 0) {
@@ -377,8 +385,8 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         uint32_t full_parity = 0;
         for (int seg = 0; seg < n_segs && ok; ++seg) {
             const int unit = u0 + seg;
-            const long long ub = (long long)unit * T;
-            const int je = (int)((ub + T < t_end ? ub + T : t_end) - t_begin);
+            const int ub = unit * T;
+            const int je = (ub + T < t_end ? ub + T : t_end) - t_begin;
 
             // ---- Q fragments (A operand): row qrow = head, 16 columns per k-step; heads >= G are zero rows
             const int qs = seg % NQ;
@@ -417,7 +425,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                     stage -= NS;
                     full_parity ^= 1u;
                 }
-                const int tile = (int)(t_begin + j - ub);
+                const int tile = t_begin + j - ub;
                 const int rows = len - tile * kStreamTile < kStreamTile ? len - tile * kStreamTile : kStreamTile;
                 const uint32_t St = ring + (uint32_t)s * TR::STAGE_BYTES;
                 if (rows > 0) {
@@ -537,7 +545,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             const int un = u0 + sg;
             page = 0;
             dev_len = len;
-            if (sg < n_segs && (long long)(un + 1) * T <= t_end) {
+            if (sg < n_segs && (un + 1) * T <= t_end) {
                 if (a.fused && len < lv.cap) {
                     const int pidx = un * lv.pages_per_unit + new_page_idx;
                     page = lv.identity_pages ? pidx : __ldg(&lv.page_table[pidx]);
@@ -549,7 +557,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         closing_loads(0, page_cur, dev_len_cur);
         for (int seg = 0; seg < n_segs && ok; ++seg, page_cur = page_nxt, dev_len_cur = dev_len_nxt) {
             const int unit = u0 + seg;
-            const long long ub = (long long)unit * T;
+            const int ub = unit * T;
             const bool opens = ub >= t_begin, closes = ub + T <= t_end;
             const int qs = seg % NQ, buf = seg % NPB;
             closing_loads(seg + 1, page_nxt, dev_len_nxt);

@@ -122,6 +122,7 @@ bool derive(const lar_config_t* c, Derived& d) {
     }
     d.max_seg = 1;
     const int t_max = (d.cap + lar::kStreamTile - 1) / lar::kStreamTile;
+    if (c->dtype == LAR_BF16 && (long long)d.units * t_max >= (1ll << 30)) return false;  // the kernel's tile indices are 32-bit
     for (int T = 1; T <= t_max; ++T) {
         const long long chunk = (long long)d.units * T / d.ctas;
         long long b = chunk >= 1 ? (T + chunk - 1) / chunk + 1 : T;
