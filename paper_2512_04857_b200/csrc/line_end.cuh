@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(128) append_kernel(const LayerView lv, const T
 __host__ __device__ inline int line_end_smem_bytes(int row_bytes, int D, int M, int total_rows, int warps, int nq, int is_bf16) {
     int b = ((M + 7) / 8 * 8) * (row_bytes + 16);  // mid keys (whole 8-key tiles), rows padded by one chunk against bank conflicts
     if (is_bf16)
-        b += ((nq + 15) / 16 * 16) * (row_bytes + 16) + M * 4;  // guide rows (whole 16-row tiles), column sums
+        b += ((nq + 15) / 16 * 16) * (row_bytes + 16) + warps * M * 4;  // guide rows (whole 16-row tiles), column sums per warp
     else
         b += warps * (D + 2 * M) * 4;      // per warp: query row (fp32), logits row, score accumulator
     b += M * 4;                            // final scores
@@ -57,7 +57,8 @@ __host__ __device__ inline int line_end_smem_bytes(int row_bytes, int D, int M, 
 }
 
 // Eq. 9 on tensor cores (bf16).  kmid: [M8][KROW] keys, qg: [nq16][KROW] guide rows (both staged, rows of KROW
-// bytes), colsum: [M] zeroed.  Every warp takes 16-row blocks of guide rows; a block's logits against all keys
+// bytes), colsum: [W][M] zeroed, one row per warp (summed in a fixed order afterwards: the scores, and with them the
+// kept sets, are reproducible from run to run).  Every warp takes 16-row blocks of guide rows; a block's logits against all keys
 // are formed twice with mma.sync m16n8k16 -- once for the row maxima and sums, once more to add the normalised
 // probabilities into the column sums -- which is cheaper than keeping a [16][M] tile of logits anywhere.
 template <int D>
@@ -122,10 +123,11 @@ __device__ __forceinline__ void score_mma(const unsigned char* kmid, const unsig
                 v0 += __shfl_xor_sync(0xffffffffu, v0, off);
                 v1 += __shfl_xor_sync(0xffffffffu, v1, off);
             }
-            if (grow == 0) {
+            if (grow == 0) {  // lanes 0..3 own two keys each of this tile in the warp's row of column sums
                 const int key = nt * 8 + 2 * quad;
-                if (key < M) atomicAdd(colsum + key, v0);
-                if (key + 1 < M) atomicAdd(colsum + key + 1, v1);
+                float* mine = colsum + warp * M;
+                if (key < M) mine[key] += v0;
+                if (key + 1 < M) mine[key + 1] += v1;
             }
         }
     }
@@ -165,9 +167,9 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv, floa
     unsigned char* kmid = smem;
     unsigned char* after_k = smem + (size_t)M8 * KROW;
     unsigned char* qg = after_k;                                                // [nq16][KROW]   (bf16)
-    float* colsum = reinterpret_cast<float*>(after_k + (size_t)nq16 * KROW);    // [M]            (bf16)
+    float* colsum = reinterpret_cast<float*>(after_k + (size_t)nq16 * KROW);    // [W][M]         (bf16)
     float* wbuf = reinterpret_cast<float*>(after_k);                            // [W][D + 2 M]   (fp32)
-    float* S = kMma ? colsum + M : wbuf + W * (D + 2 * M);
+    float* S = kMma ? colsum + W * M : wbuf + W * (D + 2 * M);
     unsigned char* keep = reinterpret_cast<unsigned char*>(S + M);
     int* srcmap = reinterpret_cast<int*>(keep + ((M + 3) / 4) * 4);
 
@@ -187,13 +189,15 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv, floa
             if (r < nq) val = *reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(gq) + (size_t)r * ROW_BYTES + c * 16);
             *reinterpret_cast<uint4*>(qg + r * KROW + c * 16) = val;
         }
-        for (int mm = tid; mm < M; mm += blockDim.x) colsum[mm] = 0.f;
+        for (int mm = tid; mm < W * M; mm += blockDim.x) colsum[mm] = 0.f;
         __syncthreads();
         score_mma<D>(kmid, qg, colsum, M, nq, scale_log2, warp, lane, W);
         __syncthreads();
         const float inv_nq = 1.f / (float)nq;
         for (int mm = tid; mm < M; mm += blockDim.x) {
-            const float sc = colsum[mm] * inv_nq;
+            float sc = 0.f;
+            for (int w = 0; w < W; ++w) sc += colsum[w * M + mm];
+            sc *= inv_nq;
             S[mm] = sc;
             lv.scores[(size_t)unit * lv.mid_pad + mm] = sc;
         }

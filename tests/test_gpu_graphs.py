@@ -58,3 +58,24 @@ def test_graph_replay_of_a_second_generation_matches_the_oracle(shape, kw, tile_
                 assert np.array_equal(pos_gpu, pos_ref), (layer, s, h)
     assert worst <= TOL[w.dtype], worst
     r.close()
+
+
+def test_two_runs_give_bit_identical_outputs_and_kept_sets():
+    """No result depends on the order in which CTAs or warps happen to finish: scores are summed in a fixed order, the
+    cross-CTA merge reads its partials in segment order."""
+    w = W.WORKLOADS["gqa_1024"].scaled(n_layers=2, batch=2, n_q_heads=8, n_kv_heads=2, n_lines=12)
+    dev = torch.device("cuda:0")
+    outs, maps = [], []
+    for tile_ranges in (False, True):
+        for _ in range(2):
+            r = bench.Runner(w, dev, _args(tile_ranges=tile_ranges))
+            r.generation()                 # eager launches
+            torch.cuda.synchronize(dev)
+            assert r.cache.poll_device_status() == 0
+            outs.append(r.out.clone())
+            maps.append([r.cache.get_state(layer)[1].copy() for layer in range(w.n_layers)])
+            r.close()
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[2], outs[3])
+    for a, b in ((maps[0], maps[1]), (maps[2], maps[3]), (maps[0], maps[2])):
+        for x, y in zip(a, b):
+            assert np.array_equal(x, y)
