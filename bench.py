@@ -182,6 +182,7 @@ class Runner:
         import torch
         from paper_2512_04857_b200 import lar, workloads as W
         self.torch, self.lar, self.w, self.dev = torch, lar, w, dev
+        self.per_layer_line_end = bool(getattr(args, "per_layer_line_end", False))
         flags = lar.LAR_FLAG_NO_HOST_CHECKS | flags_extra
         if not args.no_pdl:
             flags |= lar.LAR_FLAG_PDL
@@ -225,9 +226,12 @@ class Runner:
         w, c = self.w, self.cache
         if line == w.n_lines - 1:
             return 0
-        for layer in range(w.n_layers):
-            c.line_end_score_evict(layer)
-        return w.n_layers
+        if self.per_layer_line_end:
+            for layer in range(w.n_layers):
+                c.line_end_score_evict(layer)
+            return w.n_layers
+        c.line_end_score_evict_all()
+        return 1
 
     def capture(self):
         """Two graphs per line: A = (reset + prefill on line 0) + n x L fused decode steps, B = L line ends."""
@@ -351,7 +355,7 @@ def measure_e2e(w, dev, args, steps=1):
                         cache.decode_step_host(layer, hq[t, layer], hk[t, layer], hv[t, layer], ho[t, layer])
                 if kind == "line+end":
                     for layer in range(L):
-                        cache.line_end_score_evict(layer)
+                        cache.line_end_score_evict(layer)     # (per layer here: the host copies of a layer precede its kernels)
             graphs.append(g)
 
         def gen():
@@ -400,7 +404,8 @@ def run_ours(args):
         r = Runner(wl, dev, args, input_lines=input_lines)
         if args.eager:
             r.launches_per_generation = (wl.n_layers * (wl.n_visual + (1 if wl.cond_len else 0))
-                                         + (0 if wl.is_full_cache else wl.n_layers * (wl.n_lines - 1)))
+                                         + (0 if wl.is_full_cache else
+                                            (wl.n_layers if r.per_layer_line_end else 1) * (wl.n_lines - 1)))
         else:
             r.capture()
         sampler = ClockSampler(local) if sample_clocks else None
@@ -431,8 +436,8 @@ def run_ours(args):
                        "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
                        "storage": w.dtype, "prefix": w.cond_len, "grid": f"{w.n_lines}x{w.line_width}",
                        "budget_lines": w.budget_lines, "anchor": w.anchor_len, "recent_lines": w.recent_lines,
-                       "launch": "cuda-graph per line, fused append+decode, PDL" if not args.no_pdl
-                       else "cuda-graph per line, fused append+decode",
+                       "launch": ("cuda-graph per line, fused append+decode" + (", PDL" if not args.no_pdl else "") +
+                                  (", line end per layer" if args.per_layer_line_end else ", one line-end launch for all layers")),
                        "l2": "inputs larger than L2: all layers cycled every token "
                              f"({kv_bytes / n_decode / 1e6:.0f} MB per launch x {w.n_layers} layers)",
                        "plan": main["plan"], "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
@@ -548,6 +553,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling / small cases)")
     ap.add_argument("--eager", action="store_true", help="plain stream launches instead of CUDA graphs (profiling)")
     ap.add_argument("--no-pdl", action="store_true")
+    ap.add_argument("--per-layer-line-end", action="store_true", help="one line-end launch per layer instead of one for all layers")
     ap.add_argument("--tile-ranges", action="store_true", help="deal 32-row tiles, not whole units, to the decode CTAs")
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

@@ -164,6 +164,11 @@ lar_status_t lar_decode_step_host(lar_cache_t* c, int layer, const void* q_host,
  * [prefix | anchor | kept mid | recent], leaving an n-token buffer for the next line. */
 lar_status_t lar_line_end_score_evict(lar_cache_t* c, int layer, void* stream);
 
+/* lar_line_end_score_evict for every layer of the cache in ONE kernel launch (the line end is a synchronisation
+ * point of the whole model, Sec. 3.3; layers are independent, so their units share a grid).  Legal only when every
+ * layer has just completed the line, else LAR_ERR_BAD_STATE and nothing is launched. */
+lar_status_t lar_line_end_score_evict_all(lar_cache_t* c, void* stream);
+
 /* Destroy the host object.  The slab is the caller's and is not touched. */
 lar_status_t lar_cache_destroy(lar_cache_t* c);
 

@@ -33,6 +33,22 @@ struct LayerView {
     int identity_pages;     // 1: unit u owns pages u * pages_per_unit ... in order (the table need not be read)
 };
 
+// Byte distance between the same array of consecutive layers (a kernel whose grid spans several layers).
+struct LayerStrides {
+    size_t pool, page_table, index_map, state, guide, scores;
+};
+__host__ __device__ inline LayerView layer_view_at(LayerView lv, const LayerStrides& ls, int layers_ahead) {
+    const size_t y = (size_t)layers_ahead;
+    lv.k_pool += y * ls.pool;
+    lv.v_pool += y * ls.pool;
+    lv.page_table = reinterpret_cast<const int*>(reinterpret_cast<const char*>(lv.page_table) + y * ls.page_table);
+    lv.index_map = reinterpret_cast<int*>(reinterpret_cast<char*>(lv.index_map) + y * ls.index_map);
+    lv.state = reinterpret_cast<UnitState*>(reinterpret_cast<char*>(lv.state) + y * ls.state);
+    lv.guide += y * ls.guide;
+    lv.scores = reinterpret_cast<float*>(reinterpret_cast<char*>(lv.scores) + y * ls.scores);
+    return lv;
+}
+
 // ---------------------------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));

@@ -354,7 +354,7 @@ DecodeStreamFn decode_stream_fn(const lar_config_t& c, int G) {
     return c.head_dim == 64 ? decode_stream_for_group<64>(G) : decode_stream_for_group<128>(G);
 }
 using DecodeFn = void (*)(const lar::DecodeArgs);
-using LineEndFn = void (*)(const lar::LayerView, float);
+using LineEndFn = void (*)(const lar::LayerView, const lar::LayerStrides, float);
 
 template <typename T, int D>
 DecodeFn decode_for_group(int G) {
@@ -698,6 +698,17 @@ lar_status_t lar_decode_step_host(lar_cache_t* c, int layer, const void* q_host,
     return LAR_OK;
 }
 
+static lar::LayerStrides layer_strides(const lar_cache* c) {
+    lar::LayerStrides ls;
+    ls.pool = c->L.stride_pool;
+    ls.page_table = c->L.stride_ptab;
+    ls.index_map = c->L.stride_imap;
+    ls.state = c->L.stride_state;
+    ls.guide = c->L.stride_guide;
+    ls.scores = c->L.stride_scores;
+    return ls;
+}
+
 lar_status_t lar_line_end_score_evict(lar_cache_t* c, int layer, void* stream) {
     if (bad_layer(c, layer)) return LAR_ERR_INVALID_ARG;
     LayerShadow& sh = c->sh[layer];
@@ -707,13 +718,34 @@ lar_status_t lar_line_end_score_evict(lar_cache_t* c, int layer, void* stream) {
     if (c->d.compressing) {
         const lar::LayerView lv = view_of(c, layer);
         LineEndFn fn = line_end_fn(c->cfg, c->d.group);
-        fn<<<c->d.units, c->d.le_threads, c->plan.line_end_smem_bytes, (cudaStream_t)stream>>>(lv, c->scale * 1.4426950408889634f);
+        fn<<<dim3((unsigned)c->d.units, 1, 1), c->d.le_threads, c->plan.line_end_smem_bytes, (cudaStream_t)stream>>>(
+            lv, layer_strides(c), c->scale * 1.4426950408889634f);
         LAR_CUDA(cudaGetLastError());
         c->launches++;
         c->last_layer = layer;
         if (sh.v >= c->d.B) sh.v -= c->cfg.line_width;
     }
     sh.line_fill = 0;
+    return LAR_OK;
+}
+
+lar_status_t lar_line_end_score_evict_all(lar_cache_t* c, void* stream) {
+    if (!c) return LAR_ERR_INVALID_ARG;
+    if (c->host_checks)
+        for (const LayerShadow& sh : c->sh)
+            if (sh.pending_decode || sh.line_fill != c->cfg.line_width) return LAR_ERR_BAD_STATE;
+    if (c->d.compressing) {
+        const lar::LayerView lv = view_of(c, 0);
+        LineEndFn fn = line_end_fn(c->cfg, c->d.group);
+        fn<<<dim3((unsigned)c->d.units, (unsigned)c->cfg.n_layers, 1), c->d.le_threads, c->plan.line_end_smem_bytes,
+             (cudaStream_t)stream>>>(lv, layer_strides(c), c->scale * 1.4426950408889634f);
+        LAR_CUDA(cudaGetLastError());
+        c->launches++;
+        c->last_layer = -2;  // every layer's cache was just written: the next decode launch must not fetch ahead
+        for (LayerShadow& sh : c->sh)
+            if (sh.v >= c->d.B) sh.v -= c->cfg.line_width;
+    }
+    for (LayerShadow& sh : c->sh) sh.line_fill = 0;
     return LAR_OK;
 }
 

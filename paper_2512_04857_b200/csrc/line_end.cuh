@@ -133,10 +133,11 @@ __device__ __forceinline__ void score_mma(const unsigned char* kmid, const unsig
     }
 }
 
-// One CTA per unit.  Scoring: bf16 on tensor cores (score_mma); fp32 on CUDA cores, where every lane owns the keys
+// One CTA per unit; blockIdx.y counts layers from the one `lv0` describes (a grid may span all layers of a cache:
+// they are independent).  Scoring: bf16 on tensor cores (score_mma); fp32 on CUDA cores, where every lane owns the keys
 // m = lane, lane + 32, ... and computes whole dot products against a query row broadcast from shared memory.
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv, float scale_log2) {
+__global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, const LayerStrides ls, float scale_log2) {
     constexpr int EPL = Elt<T>::kPerChunk;
     constexpr int ROW_BYTES = D * (int)sizeof(T);
     constexpr int CHUNKS = ROW_BYTES / 16;
@@ -145,6 +146,7 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv, floa
     grid_dep_wait();
     grid_dep_launch();
 
+    const LayerView lv = layer_view_at(lv0, ls, (int)blockIdx.y);
     const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, W = blockDim.x >> 5;
     const UnitState st = lv.state[unit];
     const int C = lv.cond_len, n = lv.line_width, B = lv.budget_tokens;

@@ -68,6 +68,7 @@ def lib():
         "lar_decode_step": (C.c_int, [vp, ip, vp, vp, vp, vp, vp]),
         "lar_decode_step_host": (C.c_int, [vp, ip, vp, vp, vp, vp, vp]),
         "lar_line_end_score_evict": (C.c_int, [vp, ip, vp]),
+        "lar_line_end_score_evict_all": (C.c_int, [vp, vp]),
         "lar_cache_destroy": (C.c_int, [vp]),
         "lar_cache_get_state": (C.c_int, [vp, ip, vp, vp, vp, vp]),
         "lar_cache_poll_device_status": (C.c_int, [vp, C.POINTER(C.c_uint32), vp]),
@@ -164,6 +165,10 @@ def lar_line_end_score_evict(cache, layer, stream=None):
     _chk(lib().lar_line_end_score_evict(cache, layer, stream), "lar_line_end_score_evict")
 
 
+def lar_line_end_score_evict_all(cache, stream=None):
+    _chk(lib().lar_line_end_score_evict_all(cache, stream), "lar_line_end_score_evict_all")
+
+
 def lar_cache_destroy(cache):
     _chk(lib().lar_cache_destroy(cache), "lar_cache_destroy")
 
@@ -255,6 +260,9 @@ class Cache:
 
     def line_end_score_evict(self, layer):
         lar_line_end_score_evict(self.handle, layer, self._stream())
+
+    def line_end_score_evict_all(self):
+        lar_line_end_score_evict_all(self.handle, self._stream())
 
     def set_host_checks(self, enabled):
         lar_cache_set_host_checks(self.handle, enabled)

@@ -48,7 +48,7 @@ def pick_units(w: W.Workload, n: int, seed: int = 0) -> List[Tuple[int, int, int
 
 def run_parity(w: W.Workload, *, units: Optional[Sequence[Tuple[int, int, int]]] = None, fused: bool = True,
                gen_device: str = "cpu", n_steps: Optional[int] = None, cfg_overrides: Optional[Dict] = None,
-               check_scores: bool = True, device: str = "cuda:0") -> ParityReport:
+               check_scores: bool = True, device: str = "cuda:0", line_end_all: bool = False) -> ParityReport:
     dev = torch.device(device)
     cfg = lar.config_from_workload(w, **(cfg_overrides or {}))
     cache = lar.Cache(cfg, device=device)
@@ -116,8 +116,11 @@ def run_parity(w: W.Workload, *, units: Optional[Sequence[Tuple[int, int, int]]]
                     rep.mismatches.append(f"out layer {l} seq {s} head {h} token {t0 + t + 1}: max abs err {err:.3e}")
         # ---- line end
         if (t1 - t0) == n and t1 < w.n_visual:
-            for layer in range(L):
-                cache.line_end_score_evict(layer)
+            if line_end_all:
+                cache.line_end_score_evict_all()           # one launch for every layer
+            else:
+                for layer in range(L):
+                    cache.line_end_score_evict(layer)
             for layer in layers_sampled:
                 lens, imap, gscores = cache.get_state(layer, want_scores=True)
                 for (l, s, h) in units:

@@ -87,6 +87,27 @@ def test_small_bf16_shapes_all_units(name):
     assert rep.compressions > 0
 
 
+@pytest.mark.parametrize("name", ["janus", "gqa"])
+def test_line_end_of_all_layers_in_one_launch(name):
+    w = SMALL[name].scaled(n_layers=3)
+    rep = run_parity(w, line_end_all=True, cfg_overrides=dict(flags=lar.LAR_FLAG_PDL))
+    _check(rep, w, allow_near_ties=2)
+    assert rep.compressions > 0
+
+
+def test_line_end_of_all_layers_fp32_and_protocol():
+    w = W.WORKLOADS["tiny_b"].scaled(n_layers=2)
+    rep = run_parity(w, line_end_all=True)
+    _check(rep, w)
+    # every layer must have finished the line
+    cfg = lar.config_from_workload(w)
+    c = lar.Cache(cfg)
+    with pytest.raises(lar.LarError) as e:
+        c.line_end_score_evict_all()
+    assert e.value.status == lar.LAR_ERR_BAD_STATE
+    c.close()
+
+
 # ------------------------------------------------------------------ edge cases
 @pytest.mark.parametrize("kw", [
     dict(cond_len=0),                                        # no prefix
