@@ -567,22 +567,25 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             const uint16_t* Q16 = reinterpret_cast<const uint16_t*>(Qs);
 
             // ---- the token of this step (Eq. 4, 8): logit per head, value row, stores
-            float s_new[G], v_new[PER];
+            // Merge layout: the warp's lanes are split over the G heads, LPH lanes per head; lane (hg, sub) owns the
+            // elements sub, sub + LPH, ... of head hg (EPH of them) -- one set of exponentials per lane, not G.
+            constexpr int LPH = 32 / G, EPH = D / LPH;
+            const int hg = lane / LPH, sub = lane % LPH;
+            float s_new[G], v_new[EPH];
             const bool with_new = a.fused && closes;
 #pragma unroll
             for (int g = 0; g < G; ++g) s_new[g] = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < PER; ++i) v_new[i] = 0.f;
+            for (int i = 0; i < EPH; ++i) v_new[i] = 0.f;
             if (closes) {
                 if (with_new) {
                     const uint16_t* K16 = Q16 + G * D;
                     const uint16_t* V16 = K16 + D;
                     float kf[PER];
 #pragma unroll
-                    for (int i = 0; i < PER; ++i) {
-                        kf[i] = bf16_bits_to_float(K16[lane + 32 * i]);
-                        v_new[i] = bf16_bits_to_float(V16[lane + 32 * i]);
-                    }
+                    for (int i = 0; i < PER; ++i) kf[i] = bf16_bits_to_float(K16[lane + 32 * i]);
+#pragma unroll
+                    for (int i = 0; i < EPH; ++i) v_new[i] = bf16_bits_to_float(V16[sub + LPH * i]);
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
                         float sv = 0.f;
@@ -636,31 +639,33 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             const float* pb = pbuf + buf * pbuf_floats;
             // branch-free and unrolled over the (at most kMaxConsumers) consumer warps, so that the shared-memory
-            // loads of all heads are in flight together
-            float Mg[G], Lg[G], Og[G][PER];
+            // loads are in flight together
+            float s_mine = s_new[0];
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                float mw[kMaxConsumers], fw[kMaxConsumers];
-                float M = s_new[g];
+            for (int g = 1; g < G; ++g) s_mine = hg == g ? s_new[g] : s_mine;
+            float Mh, Lh, Oh[EPH];
+            {
+                float mw[kMaxConsumers];
+                float M = s_mine;
 #pragma unroll
                 for (int w = 0; w < kMaxConsumers; ++w) {
-                    mw[w] = w < W ? pb[(w * G + g) * PS + D] : -INFINITY;
+                    mw[w] = w < W ? pb[(w * G + hg) * PS + D] : -INFINITY;
                     M = fmaxf(M, mw[w]);
                 }
-                const float f_new = exp2_or_zero(s_new[g], M);
+                const float f_new = exp2_or_zero(s_mine, M);
                 float L = f_new;
 #pragma unroll
-                for (int i = 0; i < PER; ++i) Og[g][i] = v_new[i] * f_new;
+                for (int i = 0; i < EPH; ++i) Oh[i] = v_new[i] * f_new;
 #pragma unroll
                 for (int w = 0; w < kMaxConsumers; ++w) {
-                    const float* pw = pb + ((w < W ? w : 0) * G + g) * PS;
-                    fw[w] = exp2_or_zero(mw[w], M);
-                    L = fmaf(pw[D + 1], fw[w], L);
+                    const float* pw = pb + ((w < W ? w : 0) * G + hg) * PS;
+                    const float f = exp2_or_zero(mw[w], M);
+                    L = fmaf(pw[D + 1], f, L);
 #pragma unroll
-                    for (int i = 0; i < PER; ++i) Og[g][i] = fmaf(pw[lane + 32 * i], fw[w], Og[g][i]);
+                    for (int i = 0; i < EPH; ++i) Oh[i] = fmaf(pw[sub + LPH * i], f, Oh[i]);
                 }
-                Mg[g] = M;
-                Lg[g] = L;
+                Mh = M;
+                Lh = L;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_pempty + buf * 8);
@@ -671,13 +676,10 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
 
             if (opens && closes) {
                 // the whole unit lies in this CTA
+                const float inv = Lh > 0.f ? 1.f / Lh : 0.f;
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const float inv = Lg[g] > 0.f ? 1.f / Lg[g] : 0.f;
-#pragma unroll
-                    for (int i = 0; i < PER; ++i)
-                        outp[((size_t)unit * G + g) * D + lane + 32 * i] = __float2bfloat16_rn(Og[g][i] * inv);
-                }
+                for (int i = 0; i < EPH; ++i)
+                    outp[((size_t)unit * G + hg) * D + sub + LPH * i] = __float2bfloat16_rn(Oh[i] * inv);
             } else {
                 // the unit is shared with neighbouring CTAs: leave a partial, the last one to arrive merges
                 const int p_first = range_owner(ub, total, Pe);
@@ -688,13 +690,10 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                 }
                 float* mine = a.partials + ((size_t)unit * a.max_seg + (p - p_first)) * G * PS;
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-#pragma unroll
-                    for (int i = 0; i < PER; ++i) mine[g * PS + lane + 32 * i] = Og[g][i];
-                    if (lane == 0) {
-                        mine[g * PS + D] = Mg[g];
-                        mine[g * PS + D + 1] = Lg[g];
-                    }
+                for (int i = 0; i < EPH; ++i) mine[hg * PS + sub + LPH * i] = Oh[i];
+                if (sub == 0) {
+                    mine[hg * PS + D] = Mh;
+                    mine[hg * PS + D + 1] = Lh;
                 }
                 __threadfence();
                 __syncwarp();

@@ -119,10 +119,14 @@ def test_line_end_of_all_layers_fp32_and_protocol():
     dict(line_width=7, n_lines=9, anchor_len=7, recent_lines=1, budget_lines=3, cond_len=3),  # odd sizes
     dict(line_width=1, n_lines=40, anchor_len=1, recent_lines=2, budget_lines=6),             # 1-token lines
     dict(dtype="bf16", head_dim=64, n_q_heads=4, n_kv_heads=2),
+    dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=1),                               # bf16, G = 8
+    dict(dtype="bf16", head_dim=64, n_q_heads=8, n_kv_heads=1, flags=0x8),                     # G = 8, tile ranges
 ])
 def test_edge_shapes(kw):
+    kw = dict(kw)
+    flags = kw.pop("flags", 0)
     w = W.WORKLOADS["tiny_b"].scaled(**kw)
-    rep = run_parity(w)
+    rep = run_parity(w, cfg_overrides=dict(flags=flags, decode_ctas=5 if flags else 0))
     _check(rep, w, allow_near_ties=1)
 
 
