@@ -21,7 +21,8 @@
  *     table lists B = 96 for N = 576 at ratio 1/6, i.e. exactly rho * N).
  *   - first compression happens at the end of line B/n (cache exactly full).
  *   - N_init and r are parameters (their values are not in the paper's main text).
- *   - the softmax of Eq. 9 normalises over the mid keys only, as the equation is written.
+ *   - the softmax of Eq. 9 normalises over the mid keys only, as the equation is written
+ *     (score_norm = 1 selects the other reading: the probabilities the queries had at decode time).
  *   - with grouped-query attention the score of a cached token is the mean over the G query heads
  *     that share its KV head (folded into the 1/n of Eq. 9 as 1/(nG)).
  *   - ties in BottomK: among equal scores the token with the higher original position is evicted
@@ -50,6 +51,8 @@ typedef struct {
     int group;         /* G query heads per KV head */
     int head_dim;      /* d      */
     double scale;      /* logit scale; 0 selects 1/sqrt(d) */
+    int score_norm;    /* 0: Eq. 9 as written (softmax over the mid keys only);
+                          1: variant -- softmax over every entry the query attended to when it was decoded */
 } lar_oracle_cfg;
 
 typedef struct {
@@ -111,6 +114,39 @@ void lar_oracle_saliency(const double *Qg, int nq, const double *Kmid, int M, in
         for (int m = 0; m < M; ++m) S[m] += a[m] / den;
     }
     for (int m = 0; m < M; ++m) S[m] /= (double)nq;
+    free(a);
+}
+
+/* ---------------------------------------------------------------------------------------------
+ * Variant of Eq. 9 (the alternative reading of its softmax): each guide query is normalised over
+ * every entry it attended to when it was decoded -- all live entries whose original position does
+ * not exceed the query's own -- and the mid columns of those probabilities are averaged.  These are
+ * the attention probabilities of Eq. 2-3 accumulated over the steps of the line.
+ *   Qg [n][G][d] guide rows, query t of the line has original position first_qpos + t;
+ *   K [len][d] live keys with original positions pos[len]; mid_slot[M] slots of the mid entries.
+ * ------------------------------------------------------------------------------------------- */
+void lar_oracle_saliency_cache(const double *Qg, int n, int G, const double *K, const int *pos, int len,
+                               int d, double scale, int first_qpos, const int *mid_slot, int M,
+                               double *S) {
+    double *a = (double *)malloc(sizeof(double) * (size_t)(len > 0 ? len : 1));
+    for (int m = 0; m < M; ++m) S[m] = 0.0;
+    for (int t = 0; t < n; ++t) {
+        for (int g = 0; g < G; ++g) {
+            const double *qrow = Qg + ((size_t)t * G + g) * d;
+            double mx = -INFINITY;
+            for (int s = 0; s < len; ++s) {
+                if (pos[s] > first_qpos + t) { a[s] = -INFINITY; continue; }   /* appended after this query */
+                double x = 0.0;
+                for (int e = 0; e < d; ++e) x += qrow[e] * K[(size_t)s * d + e];
+                a[s] = x * scale;
+                if (a[s] > mx) mx = a[s];
+            }
+            double den = 0.0;
+            for (int s = 0; s < len; ++s) { a[s] = exp(a[s] - mx); den += a[s]; }
+            for (int m = 0; m < M; ++m) S[m] += a[mid_slot[m]] / den;
+        }
+    }
+    for (int m = 0; m < M; ++m) S[m] /= (double)(n * G);
     free(a);
 }
 
@@ -251,7 +287,11 @@ int lar_oracle_unit_mid_scores(const lar_oracle_unit *u, double *scores, int *mi
         mid_pos[m] = u->pos[slots[m]];
     }
     /* all n * G guide rows contribute equally: mean over the n queries and the G heads */
-    lar_oracle_saliency(u->guide, c->line_width * c->group, Kmid, M, d, cfg_scale(c), scores);
+    if (c->score_norm == 0)
+        lar_oracle_saliency(u->guide, c->line_width * c->group, Kmid, M, d, cfg_scale(c), scores);
+    else   /* query t of the line is visual token n_vis - n + t + 1, at position C + n_vis - n + t */
+        lar_oracle_saliency_cache(u->guide, c->line_width, c->group, u->K, u->pos, u->len, d, cfg_scale(c),
+                                  c->cond_len + u->n_vis - c->line_width, slots, M, scores);
     free(Kmid); free(slots);
     return M;
 }

@@ -19,7 +19,7 @@ _LIB = None
 class Cfg(C.Structure):
     _fields_ = [("cond_len", C.c_int), ("line_width", C.c_int), ("n_lines", C.c_int),
                 ("budget_lines", C.c_int), ("anchor_len", C.c_int), ("recent_lines", C.c_int),
-                ("group", C.c_int), ("head_dim", C.c_int), ("scale", C.c_double)]
+                ("group", C.c_int), ("head_dim", C.c_int), ("scale", C.c_double), ("score_norm", C.c_int)]
 
 
 def lib():
@@ -32,6 +32,9 @@ def lib():
         L.lar_oracle_attention.restype = None
         L.lar_oracle_saliency.argtypes = [dp, C.c_int, dp, C.c_int, C.c_int, C.c_double, dp]
         L.lar_oracle_saliency.restype = None
+        L.lar_oracle_saliency_cache.argtypes = [dp, C.c_int, C.c_int, dp, ip, C.c_int, C.c_int, C.c_double,
+                                                C.c_int, ip, C.c_int, dp]
+        L.lar_oracle_saliency_cache.restype = None
         L.lar_oracle_bottomk.argtypes = [dp, ip, C.c_int, C.c_int, ip]
         L.lar_oracle_bottomk.restype = None
         L.lar_oracle_unit_create.argtypes = [C.POINTER(Cfg)]
@@ -81,14 +84,14 @@ def _f64(x):
 
 
 def make_cfg(cond_len, line_width, n_lines, budget_lines, anchor_len, recent_lines, group, head_dim,
-             scale=0.0) -> Cfg:
+             scale=0.0, score_norm=0) -> Cfg:
     return Cfg(cond_len, line_width, n_lines, budget_lines, anchor_len, recent_lines, group, head_dim,
-               float(scale))
+               float(scale), int(score_norm))
 
 
 def cfg_from_workload(w) -> Cfg:
     return make_cfg(w.cond_len, w.line_width, w.n_lines, w.budget_lines, w.anchor_len, w.recent_lines,
-                    w.group, w.head_dim)
+                    w.group, w.head_dim, score_norm=1 if getattr(w, "score_norm", "mid") == "cache" else 0)
 
 
 def attention(q, K, V, scale, want_probs=False):
@@ -109,6 +112,18 @@ def saliency(Qg, Kmid, scale):
     M = Kmid.shape[0]
     S = np.zeros(M)
     lib().lar_oracle_saliency(_d(Qg), nq, _d(Kmid), M, d, float(scale), _d(S))
+    return S
+
+
+def saliency_cache(Qg, K, pos, first_qpos, mid_slot, scale):
+    """Variant of Eq. 9: Qg [n][G][d]; every query normalised over the entries it attended to."""
+    Qg, K = _f64(Qg), _f64(K)
+    n, G, d = Qg.shape
+    pos = np.ascontiguousarray(np.asarray(pos, dtype=np.int32))
+    mid_slot = np.ascontiguousarray(np.asarray(mid_slot, dtype=np.int32))
+    S = np.zeros(len(mid_slot))
+    lib().lar_oracle_saliency_cache(_d(Qg), n, G, _d(K), _i(pos), K.shape[0], d, float(scale), int(first_qpos),
+                                    _i(mid_slot), len(mid_slot), _d(S))
     return S
 
 

@@ -55,6 +55,7 @@ class Workload:
     seed: int
     prefix_key_scale: float = 1.0
     note: str = ""
+    score_norm: str = "mid"  # softmax of Eq. 9 over the "mid" keys (as written) or over the whole live "cache" (variant)
 
     @property
     def n_visual(self) -> int:            # N

@@ -320,3 +320,85 @@ def test_run_units_matches_stepwise_driver():
         for li, (_, ev, pos) in enumerate(events):
             row = kept[ui, li]
             assert list(row[row >= 0]) == list(pos)
+
+
+# ------------------------------------------------- variant of Eq. 9: normalised over the whole live cache
+def _drive_one_line(cfg, seed, want_probs):
+    """Prefill, run to the first compressing line end; returns the unit and the last line's step probabilities."""
+    r = np.random.default_rng(seed)
+    C_, n, G, d = cfg.cond_len, cfg.line_width, cfg.group, cfg.head_dim
+    u = O.Unit(cfg)
+    u.prefill(r.normal(size=(C_, d)), r.normal(size=(C_, d)))
+    probs = []
+    for i in range(cfg.budget_lines * n):
+        res = u.step(r.normal(size=(G, d)), r.normal(size=d), r.normal(size=d), want_probs=want_probs)
+        if want_probs and i >= (cfg.budget_lines - 1) * n:
+            probs.append(res[1])
+        if (i + 1) % n == 0 and (i + 1) < cfg.budget_lines * n:
+            assert u.line_end() is None
+    assert u.line_end_due() == 1
+    return u, probs
+
+
+@pytest.mark.parametrize("G", [1, 3])
+def test_cache_normalised_scores_are_the_decode_probabilities_of_the_line(G):
+    # the variant's score of a mid token = mean over the line's steps and heads of the probability Eq. 2-3 gave it
+    # at that step (those probabilities are pinned to the library softmax above)
+    cfg = O.make_cfg(5, 6, 10, 5, 4, 2, G, 16, score_norm=1)
+    u, probs = _drive_one_line(cfg, 77, True)
+    S, mid_pos = u.mid_scores()
+    pos = u.positions()
+    slot_of = {int(p): s for s, p in enumerate(pos)}
+    expect = np.zeros(len(mid_pos))
+    for p_t in probs:                       # [G][len at that step]; slots do not move within a line
+        for m, mp in enumerate(mid_pos):
+            expect[m] += p_t[:, slot_of[int(mp)]].sum()
+    expect /= cfg.line_width * G
+    np.testing.assert_allclose(S, expect, rtol=1e-12, atol=1e-15)
+    assert 0.0 < S.sum() < 1.0              # the mid region holds only part of every query's mass
+
+
+def test_cache_normalised_scores_vs_library_softmax_with_causal_cut():
+    r = np.random.default_rng(5)
+    n, G, d, ln = 4, 2, 8, 19
+    Qg, K = r.normal(size=(n, G, d)), r.normal(size=(ln, d))
+    pos = np.arange(ln) + 3                 # any increasing positions
+    first_qpos = int(pos[ln - n])
+    mid = [2, 3, 5, 6, 7, 9]
+    S = O.saliency_cache(Qg, K, pos, first_qpos, mid, 0.3)
+    expect = np.zeros(len(mid))
+    for t in range(n):
+        live = ln - n + t + 1               # entries appended up to and including query t's own token
+        for g in range(G):
+            expect += sp_softmax((K[:live] @ Qg[t, g]) * 0.3)[mid]
+    np.testing.assert_allclose(S, expect / (n * G), rtol=1e-12, atol=1e-15)
+
+
+def test_cache_normalisation_reduces_to_eq9_when_only_the_mid_keys_carry_mass():
+    # every key outside the mid region points away from all queries with a huge norm: its probability underflows
+    # to zero and the two readings of Eq. 9 coincide
+    r = np.random.default_rng(9)
+    n, G, d, ln = 3, 2, 6, 14
+    Qg = np.abs(r.normal(size=(n, G, d)))
+    K = r.normal(size=(ln, d))
+    mid = [4, 5, 6, 7, 8]
+    for s in range(ln):
+        if s not in mid:
+            K[s] = -1e3
+    pos = np.arange(ln)
+    a = O.saliency_cache(Qg, K, pos, ln - n, mid, 1.0)
+    b = O.saliency(Qg.reshape(n * G, d), K[mid], 1.0)
+    np.testing.assert_allclose(a, b, rtol=1e-12)
+    assert abs(a.sum() - 1.0) < 1e-9
+
+
+def test_the_two_normalisations_differ_and_can_change_the_kept_set():
+    cfg0 = O.make_cfg(5, 6, 10, 5, 4, 2, 2, 16, score_norm=0)
+    cfg1 = O.make_cfg(5, 6, 10, 5, 4, 2, 2, 16, score_norm=1)
+    u0, _ = _drive_one_line(cfg0, 3, False)
+    u1, _ = _drive_one_line(cfg1, 3, False)
+    S0, p0 = u0.mid_scores()
+    S1, p1 = u1.mid_scores()
+    assert (p0 == p1).all()
+    assert abs(S0.sum() - 1.0) < 1e-9 and S1.sum() < 0.9
+    assert not np.allclose(S0 / S0.sum(), S1 / S1.sum(), rtol=1e-3)
