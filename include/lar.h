@@ -65,6 +65,13 @@ typedef enum { LAR_BF16 = 0, LAR_FP32 = 1 } lar_dtype_t;
 #define LAR_FLAG_SHUFFLE_PAGES 0x4u  /* test hook: assign physical pages in a pseudo-random order */
 #define LAR_FLAG_TILE_RANGES 0x8u    /* bf16 decode: always deal 32-row tiles (not whole units) to the CTAs, even
                                         where whole units would balance well enough */
+#define LAR_FLAG_SCORE_CACHE_NORM 0x10u /* variant of Eq. 9 (Sec. 3.3): the softmax of every guide query runs over
+                                        all entries that were live when its token was decoded (conditional,
+                                        anchor, mid, recent and the line's own tokens up to itself) instead of
+                                        over the mid keys only; the score of a mid token is then the attention
+                                        probability Eq. 2-3 gave it, averaged over the n steps of the line and
+                                        the G heads.  The line-end kernel stages C + B keys in shared memory:
+                                        configurations where they do not fit are rejected at creation. */
 
 typedef struct lar_config {
     uint32_t struct_size;  /* = sizeof(lar_config_t) */

@@ -238,7 +238,8 @@ lar_status_t plan_query_impl(const lar_config_t* cfg, lar_plan_t* out, Derived* 
     choose_plan(cfg, d, p);
     p.line_end_smem_bytes =
         d.compressing ? lar::line_end_smem_bytes(d.row_bytes, cfg->head_dim, d.M, d.M - cfg->line_width + cfg->recent_lines * cfg->line_width, d.le_threads / 32,
-                                                 cfg->line_width * d.group, cfg->dtype == LAR_BF16 ? 1 : 0) : 0;
+                                                 cfg->line_width * d.group, cfg->dtype == LAR_BF16 ? 1 : 0, cfg->cond_len + d.B,
+                                                 (cfg->flags & LAR_FLAG_SCORE_CACHE_NORM) ? 1 : 0) : 0;
     p.slab_bytes = L.total;
     p.scratch_bytes = (L.off_tickets + L.tickets_bytes) - L.off_partials;
     if (p.decode_smem_bytes > 227 * 1024 || p.line_end_smem_bytes > 227 * 1024) return LAR_ERR_INVALID_ARG;
@@ -354,7 +355,7 @@ DecodeStreamFn decode_stream_fn(const lar_config_t& c, int G) {
     return c.head_dim == 64 ? decode_stream_for_group<64>(G) : decode_stream_for_group<128>(G);
 }
 using DecodeFn = void (*)(const lar::DecodeArgs);
-using LineEndFn = void (*)(const lar::LayerView, const lar::LayerStrides, float);
+using LineEndFn = void (*)(const lar::LayerView, const lar::LayerStrides, float, int);
 
 template <typename T, int D>
 DecodeFn decode_for_group(int G) {
@@ -719,7 +720,7 @@ lar_status_t lar_line_end_score_evict(lar_cache_t* c, int layer, void* stream) {
         const lar::LayerView lv = view_of(c, layer);
         LineEndFn fn = line_end_fn(c->cfg, c->d.group);
         fn<<<dim3((unsigned)c->d.units, 1, 1), c->d.le_threads, c->plan.line_end_smem_bytes, (cudaStream_t)stream>>>(
-            lv, layer_strides(c), c->scale * 1.4426950408889634f);
+            lv, layer_strides(c), c->scale * 1.4426950408889634f, (c->cfg.flags & LAR_FLAG_SCORE_CACHE_NORM) ? 1 : 0);
         LAR_CUDA(cudaGetLastError());
         c->launches++;
         c->last_layer = layer;
@@ -738,7 +739,8 @@ lar_status_t lar_line_end_score_evict_all(lar_cache_t* c, void* stream) {
         const lar::LayerView lv = view_of(c, 0);
         LineEndFn fn = line_end_fn(c->cfg, c->d.group);
         fn<<<dim3((unsigned)c->d.units, (unsigned)c->cfg.n_layers, 1), c->d.le_threads, c->plan.line_end_smem_bytes,
-             (cudaStream_t)stream>>>(lv, layer_strides(c), c->scale * 1.4426950408889634f);
+             (cudaStream_t)stream>>>(lv, layer_strides(c), c->scale * 1.4426950408889634f,
+                                     (c->cfg.flags & LAR_FLAG_SCORE_CACHE_NORM) ? 1 : 0);
         LAR_CUDA(cudaGetLastError());
         c->launches++;
         c->last_layer = -2;  // every layer's cache was just written: the next decode launch must not fetch ahead

@@ -44,59 +44,89 @@ __global__ void __launch_bounds__(128) append_kernel(const LayerView lv, const T
 // ------------------------------------------------------------------------------------- line end
 // Shared memory of line_end_kernel (bytes): M mid keys, nq = n * G guide rows, W warps.
 // bf16 (tensor-core scoring): the guide rows are staged next to the keys; fp32: per-warp row buffers.
-__host__ __device__ inline int line_end_smem_bytes(int row_bytes, int D, int M, int total_rows, int warps, int nq, int is_bf16) {
-    int b = ((M + 7) / 8 * 8) * (row_bytes + 16);  // mid keys (whole 8-key tiles), rows padded by one chunk against bank conflicts
+// cache_norm (the softmax of Eq. 9 taken over the whole live cache): all live_rows = C + B keys are staged, plus one
+// cleared 8-key tile behind them; the bf16 path then reads the guide rows straight from global memory.
+__host__ __device__ inline int line_end_staged_rows(int M, int live_rows, int cache_norm) {
+    return cache_norm ? (live_rows + 7) / 8 * 8 + 8 : (M + 7) / 8 * 8;
+}
+__host__ __device__ inline int line_end_smem_bytes(int row_bytes, int D, int M, int total_rows, int warps, int nq, int is_bf16,
+                                                   int live_rows, int cache_norm) {
+    int b = line_end_staged_rows(M, live_rows, cache_norm) * (row_bytes + 16);  // keys, rows padded by one chunk against bank conflicts
     if (is_bf16)
-        b += ((nq + 15) / 16 * 16) * (row_bytes + 16) + warps * M * 4;  // guide rows (whole 16-row tiles), column sums per warp
+        b += (cache_norm ? 0 : ((nq + 15) / 16 * 16) * (row_bytes + 16)) + warps * M * 4;  // guide rows (whole 16-row tiles), column sums per warp
     else
-        b += warps * (D + 2 * M) * 4;      // per warp: query row (fp32), logits row, score accumulator
+        b += warps * (D + (cache_norm ? live_rows : M) + M) * 4;  // per warp: query row (fp32), logits row, score accumulator
     b += M * 4;                            // final scores
     b += ((M + 3) / 4) * 4;                // keep flags
     b += total_rows * 4;                   // source slot of every surviving row
     return (b + 15) / 16 * 16 + 16;
 }
 
-// Eq. 9 on tensor cores (bf16).  kmid: [M8][KROW] keys, qg: [nq16][KROW] guide rows (both staged, rows of KROW
-// bytes), colsum: [W][M] zeroed, one row per warp (summed in a fixed order afterwards: the scores, and with them the
-// kept sets, are reproducible from run to run).  Every warp takes 16-row blocks of guide rows; a block's logits against all keys
-// are formed twice with mma.sync m16n8k16 -- once for the row maxima and sums, once more to add the normalised
-// probabilities into the column sums -- which is cheaper than keeping a [16][M] tile of logits anywhere.
-template <int D>
-__device__ __forceinline__ void score_mma(const unsigned char* kmid, const unsigned char* qg, float* colsum, int M, int nq,
-                                          float scale_log2, int warp, int lane, int W) {
+// Eq. 9 on tensor cores (bf16).  keys: staged key rows of KROW bytes, colsum: [W][M] zeroed, one row per warp (summed
+// in a fixed order afterwards: the scores, and with them the kept sets, are reproducible from run to run).  Every warp
+// takes 16-row blocks of guide rows; a block's logits are formed twice with mma.sync m16n8k16 -- once for the row
+// maxima and sums, once more to add the normalised probabilities into the column sums -- which is cheaper than
+// keeping a [16][M] tile of logits anywhere.
+//   CACHE = false: the rows are normalised over the M mid keys (keys = those M rows; guide rows staged at qg).
+//   CACHE = true:  keys holds all n_keys live rows, the mid ones from row mid_off; guide row (t, g) is normalised over
+//                  the keys that were live when token t of the line was decoded (rows < n_keys - n + t + 1) and read
+//                  from global memory (gq32: rows of D / 2 words).
+template <int D, bool CACHE>
+__device__ __forceinline__ void score_mma(const unsigned char* keys, const unsigned char* qg, const uint32_t* gq32, float* colsum,
+                                          int n_keys, int mid_off, int M, int nq, int G, int n, float scale_log2, int warp,
+                                          int lane, int W) {
     constexpr int KROW = D * 2 + 16;
     constexpr int KSTEPS = D / 16;
     const int quad = lane & 3, grow = lane >> 2;
-    const int n_tiles = (M + 7) / 8;
-    const uint32_t kbase = smem_u32(kmid), qbase = smem_u32(qg);
+    const uint32_t kbase = smem_u32(keys), qbase = smem_u32(qg);
     for (int rb = warp; rb * 16 < nq; rb += W) {
+        const int r0 = rb * 16 + grow, r1 = r0 + 8;
         uint32_t a[KSTEPS][4];
 #pragma unroll
-        for (int ks = 0; ks < KSTEPS; ++ks)
-            ldmatrix_x4(qbase + (uint32_t)((rb * 16 + (lane & 15)) * KROW + (2 * ks + (lane >> 4)) * 16), a[ks]);
-        auto logits = [&](int nt, float (&c)[4]) {
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+            if constexpr (CACHE) {
+                a[ks][0] = r0 < nq ? __ldg(gq32 + (size_t)r0 * (D / 2) + ks * 8 + quad) : 0u;
+                a[ks][1] = r1 < nq ? __ldg(gq32 + (size_t)r1 * (D / 2) + ks * 8 + quad) : 0u;
+                a[ks][2] = r0 < nq ? __ldg(gq32 + (size_t)r0 * (D / 2) + ks * 8 + 4 + quad) : 0u;
+                a[ks][3] = r1 < nq ? __ldg(gq32 + (size_t)r1 * (D / 2) + ks * 8 + 4 + quad) : 0u;
+            } else {
+                ldmatrix_x4(qbase + (uint32_t)((rb * 16 + (lane & 15)) * KROW + (2 * ks + (lane >> 4)) * 16), a[ks]);
+            }
+        }
+        // logits of the block against the 8 keys from staged row `row0`, scaled; this thread: keys 2 quad, 2 quad + 1
+        auto logits = [&](int row0, float (&c)[4]) {
             c[0] = c[1] = c[2] = c[3] = 0.f;
 #pragma unroll
             for (int i = 0; i < KSTEPS / 2; ++i) {
                 uint32_t b[4];
-                ldmatrix_x4(kbase + (uint32_t)((nt * 8 + (lane & 7)) * KROW + (4 * i + (lane >> 3)) * 16), b);
+                ldmatrix_x4(kbase + (uint32_t)((row0 + (lane & 7)) * KROW + (4 * i + (lane >> 3)) * 16), b);
                 mma_bf16(c, a[2 * i][0], a[2 * i][1], a[2 * i][2], a[2 * i][3], b[0], b[1]);
                 mma_bf16(c, a[2 * i + 1][0], a[2 * i + 1][1], a[2 * i + 1][2], a[2 * i + 1][3], b[2], b[3]);
             }
-            const int key = nt * 8 + 2 * quad;
-            c[0] = key < M ? c[0] * scale_log2 : -INFINITY;
-            c[2] = key < M ? c[2] * scale_log2 : -INFINITY;
-            c[1] = key + 1 < M ? c[1] * scale_log2 : -INFINITY;
-            c[3] = key + 1 < M ? c[3] * scale_log2 : -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) c[i] *= scale_log2;
         };
-        // pass 1: maximum and sum of every row (rows grow and grow + 8 of the block; this thread's columns first)
+        // keys every row of this thread is normalised over
+        int lim0 = n_keys, lim1 = n_keys;
+        if constexpr (CACHE) {
+            lim0 = min(n_keys, n_keys - n + r0 / G + 1);
+            lim1 = min(n_keys, n_keys - n + r1 / G + 1);
+        }
+        // pass 1: maximum and sum of every row (rows grow and grow + 8 of the block; this thread's columns first);
+        // a thread that has seen no key of a row yet keeps (-inf, 0) -- the reference point 0 avoids inf - inf
         float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-        for (int nt = 0; nt < n_tiles; ++nt) {
+        for (int k0 = 0; k0 < n_keys; k0 += 8) {
             float c[4];
-            logits(nt, c);
+            logits(k0, c);
+            const int key = k0 + 2 * quad;
+            c[0] = key < lim0 ? c[0] : -INFINITY;
+            c[1] = key + 1 < lim0 ? c[1] : -INFINITY;
+            c[2] = key < lim1 ? c[2] : -INFINITY;
+            c[3] = key + 1 < lim1 ? c[3] : -INFINITY;
             const float n0 = fmaxf(m0, fmaxf(c[0], c[1])), n1 = fmaxf(m1, fmaxf(c[2], c[3]));
-            l0 = l0 * exp2f(m0 - n0) + exp2f(c[0] - n0) + exp2f(c[1] - n0);
-            l1 = l1 * exp2f(m1 - n1) + exp2f(c[2] - n1) + exp2f(c[3] - n1);
+            const float f0 = n0 == -INFINITY ? 0.f : n0, f1 = n1 == -INFINITY ? 0.f : n1;
+            l0 = l0 * exp2f(m0 - f0) + exp2f(c[0] - f0) + exp2f(c[1] - f0);
+            l1 = l1 * exp2f(m1 - f1) + exp2f(c[2] - f1) + exp2f(c[3] - f1);
             m0 = n0;
             m1 = n1;
         }
@@ -105,17 +135,18 @@ __device__ __forceinline__ void score_mma(const unsigned char* kmid, const unsig
             const float om0 = __shfl_xor_sync(0xffffffffu, m0, off), ol0 = __shfl_xor_sync(0xffffffffu, l0, off);
             const float om1 = __shfl_xor_sync(0xffffffffu, m1, off), ol1 = __shfl_xor_sync(0xffffffffu, l1, off);
             const float n0 = fmaxf(m0, om0), n1 = fmaxf(m1, om1);
-            l0 = l0 * exp2f(m0 - n0) + ol0 * exp2f(om0 - n0);
-            l1 = l1 * exp2f(m1 - n1) + ol1 * exp2f(om1 - n1);
+            const float f0 = n0 == -INFINITY ? 0.f : n0, f1 = n1 == -INFINITY ? 0.f : n1;
+            l0 = l0 * exp2f(m0 - f0) + ol0 * exp2f(om0 - f0);
+            l1 = l1 * exp2f(m1 - f1) + ol1 * exp2f(om1 - f1);
             m0 = n0;
             m1 = n1;
         }
         // rows beyond the queue (the last block may be ragged) carry no weight
-        const float w0 = rb * 16 + grow < nq ? 1.f / l0 : 0.f, w1 = rb * 16 + grow + 8 < nq ? 1.f / l1 : 0.f;
-        // pass 2: probabilities, summed over the block's rows, into the column sums
-        for (int nt = 0; nt < n_tiles; ++nt) {
+        const float w0 = r0 < nq ? 1.f / l0 : 0.f, w1 = r1 < nq ? 1.f / l1 : 0.f;
+        // pass 2: probabilities of the mid keys, summed over the block's rows, into the column sums
+        for (int k0 = 0; k0 < M; k0 += 8) {
             float c[4];
-            logits(nt, c);
+            logits(mid_off + k0, c);
             float v0 = (w0 != 0.f ? exp2f(c[0] - m0) * w0 : 0.f) + (w1 != 0.f ? exp2f(c[2] - m1) * w1 : 0.f);
             float v1 = (w0 != 0.f ? exp2f(c[1] - m0) * w0 : 0.f) + (w1 != 0.f ? exp2f(c[3] - m1) * w1 : 0.f);
 #pragma unroll
@@ -124,7 +155,7 @@ __device__ __forceinline__ void score_mma(const unsigned char* kmid, const unsig
                 v1 += __shfl_xor_sync(0xffffffffu, v1, off);
             }
             if (grow == 0) {  // lanes 0..3 own two keys each of this tile in the warp's row of column sums
-                const int key = nt * 8 + 2 * quad;
+                const int key = k0 + 2 * quad;
                 float* mine = colsum + warp * M;
                 if (key < M) mine[key] += v0;
                 if (key + 1 < M) mine[key + 1] += v1;
@@ -134,10 +165,11 @@ __device__ __forceinline__ void score_mma(const unsigned char* kmid, const unsig
 }
 
 // One CTA per unit; blockIdx.y counts layers from the one `lv0` describes (a grid may span all layers of a cache:
-// they are independent).  Scoring: bf16 on tensor cores (score_mma); fp32 on CUDA cores, where every lane owns the keys
+// they are independent).  cache_norm != 0 selects the variant of Eq. 9 whose softmax runs over the whole live cache
+// (every guide query over the entries that were live when it was decoded).  Scoring: bf16 on tensor cores (score_mma); fp32 on CUDA cores, where every lane owns the keys
 // m = lane, lane + 32, ... and computes whole dot products against a query row broadcast from shared memory.
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, const LayerStrides ls, float scale_log2) {
+__global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, const LayerStrides ls, float scale_log2, int cache_norm) {
     constexpr int EPL = Elt<T>::kPerChunk;
     constexpr int ROW_BYTES = D * (int)sizeof(T);
     constexpr int CHUNKS = ROW_BYTES / 16;
@@ -165,35 +197,45 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
     const int nq = n * G;
 
     constexpr bool kMma = sizeof(T) == 2;  // bf16: tensor-core scoring; fp32: CUDA cores
-    const int M8 = (M + 7) / 8 * 8, nq16 = (nq + 15) / 16 * 16;
-    unsigned char* kmid = smem;
-    unsigned char* after_k = smem + (size_t)M8 * KROW;
-    unsigned char* qg = after_k;                                                // [nq16][KROW]   (bf16)
-    float* colsum = reinterpret_cast<float*>(after_k + (size_t)nq16 * KROW);    // [W][M]         (bf16)
-    float* wbuf = reinterpret_cast<float*>(after_k);                            // [W][D + 2 M]   (fp32)
-    float* S = kMma ? colsum + W * M : wbuf + W * (D + 2 * M);
+    const int nq16 = (nq + 15) / 16 * 16;
+    const int stage0 = cache_norm ? 0 : mid0;          // first staged slot
+    const int n_stage = cache_norm ? st.len : M;       // staged keys
+    const int mid_off = mid0 - stage0;                 // staged row of the first mid key
+    const int rows_pad = line_end_staged_rows(M, st.len, cache_norm);
+    unsigned char* kst = smem;
+    unsigned char* after_k = smem + (size_t)rows_pad * KROW;
+    unsigned char* qg = after_k;                                                // [nq16][KROW]   (bf16, mid-only scoring)
+    float* colsum = reinterpret_cast<float*>(after_k + (cache_norm ? (size_t)0 : (size_t)nq16 * KROW));  // [W][M] (bf16)
+    const int wstride = D + n_stage + M;
+    float* wbuf = reinterpret_cast<float*>(after_k);                            // [W][D + n_stage + M]   (fp32)
+    float* S = kMma ? colsum + W * M : wbuf + W * wstride;
     unsigned char* keep = reinterpret_cast<unsigned char*>(S + M);
     int* srcmap = reinterpret_cast<int*>(keep + ((M + 3) / 4) * 4);
 
-    // ---- stage the mid keys (rows of the last, ragged 8-key tile are cleared)
-    for (int idx = tid; idx < M8 * CHUNKS; idx += blockDim.x) {
+    // ---- stage the keys (rows behind the last one are cleared)
+    for (int idx = tid; idx < rows_pad * CHUNKS; idx += blockDim.x) {
         const int r = idx / CHUNKS, c = idx - r * CHUNKS;
         uint4 val = make_uint4(0u, 0u, 0u, 0u);
-        if (r < M) val = *reinterpret_cast<const uint4*>(lv.k_pool + row_offset(lv, unit, mid0 + r, ROW_BYTES) + c * 16);
-        *reinterpret_cast<uint4*>(kmid + r * KROW + c * 16) = val;
+        if (r < n_stage) val = *reinterpret_cast<const uint4*>(lv.k_pool + row_offset(lv, unit, stage0 + r, ROW_BYTES) + c * 16);
+        *reinterpret_cast<uint4*>(kst + r * KROW + c * 16) = val;
     }
     const T* gq = reinterpret_cast<const T*>(lv.guide) + (size_t)unit * nq * D;
     if constexpr (kMma) {
-        // ---- Eq. 9 on tensor cores: stage the guide rows, clear the column sums
-        for (int idx = tid; idx < nq16 * CHUNKS; idx += blockDim.x) {
-            const int r = idx / CHUNKS, c = idx - r * CHUNKS;
-            uint4 val = make_uint4(0u, 0u, 0u, 0u);
-            if (r < nq) val = *reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(gq) + (size_t)r * ROW_BYTES + c * 16);
-            *reinterpret_cast<uint4*>(qg + r * KROW + c * 16) = val;
+        // ---- Eq. 9 on tensor cores: stage the guide rows (mid-only scoring), clear the column sums
+        if (!cache_norm) {
+            for (int idx = tid; idx < nq16 * CHUNKS; idx += blockDim.x) {
+                const int r = idx / CHUNKS, c = idx - r * CHUNKS;
+                uint4 val = make_uint4(0u, 0u, 0u, 0u);
+                if (r < nq) val = *reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(gq) + (size_t)r * ROW_BYTES + c * 16);
+                *reinterpret_cast<uint4*>(qg + r * KROW + c * 16) = val;
+            }
         }
         for (int mm = tid; mm < W * M; mm += blockDim.x) colsum[mm] = 0.f;
         __syncthreads();
-        score_mma<D>(kmid, qg, colsum, M, nq, scale_log2, warp, lane, W);
+        if (cache_norm)
+            score_mma<D, true>(kst, qg, reinterpret_cast<const uint32_t*>(gq), colsum, n_stage, mid_off, M, nq, G, n, scale_log2, warp, lane, W);
+        else
+            score_mma<D, false>(kst, qg, nullptr, colsum, n_stage, mid_off, M, nq, G, n, scale_log2, warp, lane, W);
         __syncthreads();
         const float inv_nq = 1.f / (float)nq;
         for (int mm = tid; mm < M; mm += blockDim.x) {
@@ -205,10 +247,11 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
         }
         __syncthreads();
     } else {
-        // ---- Eq. 9 on CUDA cores: every guide row is soft-maxed over the M mid keys; rows are summed per key
-        float* qrow = wbuf + warp * (D + 2 * M);
+        // ---- Eq. 9 on CUDA cores: every guide row is soft-maxed over its keys (the M mid keys, or the entries that
+        // were live when its token was decoded); the mid columns of the rows are summed per key
+        float* qrow = wbuf + warp * wstride;
         float* logit = qrow + D;
-        float* sacc = logit + M;
+        float* sacc = logit + n_stage;
         for (int mm = lane; mm < M; mm += 32) sacc[mm] = 0.f;
         __syncthreads();
         for (int j = warp; j < nq; j += W) {
@@ -220,9 +263,10 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
                 for (int e = 0; e < EPL; ++e) qrow[c * EPL + e] = f[e] * scale_log2;
             }
             __syncwarp();
+            const int lim = cache_norm ? n_stage - n + j / G + 1 : n_stage;
             float mx = -INFINITY;
-            for (int mm = lane; mm < M; mm += 32) {
-                const unsigned char* kr = kmid + mm * KROW;
+            for (int kk = lane; kk < lim; kk += 32) {
+                const unsigned char* kr = kst + kk * KROW;
                 float acc = 0.f;
 #pragma unroll 4
                 for (int c = 0; c < CHUNKS; ++c) {
@@ -231,26 +275,27 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
 #pragma unroll
                     for (int e = 0; e < EPL; ++e) acc = fmaf(qrow[c * EPL + e], kf[e], acc);
                 }
-                logit[mm] = acc;
+                logit[kk] = acc;
                 mx = fmaxf(mx, acc);
             }
             mx = warp_max(mx);
             float sum = 0.f;
-            for (int mm = lane; mm < M; mm += 32) {
-                const float p = exp2f(logit[mm] - mx);
-                logit[mm] = p;
+            for (int kk = lane; kk < lim; kk += 32) {
+                const float p = exp2f(logit[kk] - mx);
+                logit[kk] = p;
                 sum += p;
             }
             sum = warp_sum(sum);
             const float inv = 1.f / sum;
-            for (int mm = lane; mm < M; mm += 32) sacc[mm] = fmaf(logit[mm], inv, sacc[mm]);
+            __syncwarp();
+            for (int mm = lane; mm < M; mm += 32) sacc[mm] = fmaf(logit[mid_off + mm], inv, sacc[mm]);
             __syncwarp();
         }
         __syncthreads();
         const float inv_nq = 1.f / (float)nq;
         for (int mm = tid; mm < M; mm += blockDim.x) {
             float sc = 0.f;
-            for (int w = 0; w < W; ++w) sc += wbuf[w * (D + 2 * M) + D + M + mm];
+            for (int w = 0; w < W; ++w) sc += wbuf[w * wstride + D + n_stage + mm];
             sc *= inv_nq;
             S[mm] = sc;
             lv.scores[(size_t)unit * lv.mid_pad + mm] = sc;

@@ -17,6 +17,7 @@ LAR_OK, LAR_ERR_INVALID_ARG, LAR_ERR_BAD_STATE, LAR_ERR_CAPACITY, LAR_ERR_CUDA, 
     LAR_ERR_DEVICE_CHECK = range(7)
 LAR_BF16, LAR_FP32 = 0, 1
 LAR_FLAG_NO_HOST_CHECKS, LAR_FLAG_PDL, LAR_FLAG_SHUFFLE_PAGES, LAR_FLAG_TILE_RANGES = 0x1, 0x2, 0x4, 0x8
+LAR_FLAG_SCORE_CACHE_NORM = 0x10
 
 
 class lar_config_t(C.Structure):
@@ -102,6 +103,8 @@ def config_from_workload(w, **overrides) -> lar_config_t:
               n_lines=w.n_lines, anchor_len=w.anchor_len, recent_lines=w.recent_lines,
               budget_lines=w.budget_lines)
     kw.update(overrides)
+    if getattr(w, "score_norm", "mid") == "cache":
+        kw["flags"] = kw.get("flags", 0) | LAR_FLAG_SCORE_CACHE_NORM
     return make_config(**kw)
 
 

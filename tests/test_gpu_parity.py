@@ -166,3 +166,53 @@ def test_generator_gpu_matches_cpu():
     for x, y in zip(a, b):
         diff = (x.float() != y.float().cpu()).float().mean().item()
         assert diff < 1e-4
+
+
+# ------------------------------------------------------------------ Eq. 9 normalised over the whole live cache (variant)
+@pytest.mark.parametrize("kw", [
+    dict(),                                                   # fp32, M = 48
+    dict(n_q_heads=8, n_kv_heads=1),                          # fp32, G = 8
+    dict(cond_len=0, anchor_len=0),                           # nothing in front of the mid region
+    dict(line_width=7, n_lines=9, anchor_len=7, recent_lines=1, budget_lines=3, cond_len=3),  # odd sizes, mid_off not a multiple of 8
+    dict(line_width=1, n_lines=40, anchor_len=1, recent_lines=2, budget_lines=6),             # 1-token lines
+    dict(dtype="bf16", head_dim=64, n_q_heads=4, n_kv_heads=2),
+    dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=1),
+    dict(dtype="bf16", head_dim=64, n_q_heads=4, n_kv_heads=4, cond_len=3, anchor_len=5, recent_lines=2, budget_lines=5),
+])
+def test_cache_normalised_scoring(kw):
+    w = W.WORKLOADS["tiny_b"].scaled(score_norm="cache", **kw)
+    rep = run_parity(w)
+    _check(rep, w, allow_near_ties=1)
+    assert rep.compressions > 0
+    assert rep.max_score_rel_err < (2e-3 if w.dtype == "bf16" else 1e-4)
+
+
+def test_cache_normalised_scoring_one_launch_for_all_layers():
+    """The flag must reach the kernel on the all-layers launch too: the exported scores match the oracle's variant
+    (whose scores of a unit sum to well below one, unlike Eq. 9 as written)."""
+    w = W.WORKLOADS["tiny_b"].scaled(score_norm="cache")
+    cfg = lar.config_from_workload(w)
+    assert cfg.flags & lar.LAR_FLAG_SCORE_CACHE_NORM
+    rep = run_parity(w, line_end_all=True)
+    _check(rep, w, allow_near_ties=1)
+    assert rep.max_score_rel_err < 1e-4
+
+
+@pytest.mark.parametrize("name,layers,n_units", [("janus_pro_7b", 2, 4), ("gqa_1024", 1, 3)])
+def test_cache_normalised_scoring_full_size_sampled(name, layers, n_units):
+    w = W.WORKLOADS[name].scaled(n_layers=layers, score_norm="cache")
+    rep = run_parity(w, units=pick_units(w, n_units, seed=3), gen_device="cuda", cfg_overrides=dict(flags=lar.LAR_FLAG_PDL),
+                     line_end_all=True)
+    _check(rep, w, allow_near_ties=2)
+    assert rep.compressions == n_units * (w.n_lines - w.budget_lines)
+
+
+def test_bf16_mid_region_smaller_than_one_key_tile():
+    # M = 6 < 8: some lanes of the scoring warp see no valid key at all in the only tile
+    w = W.WORKLOADS["tiny_b"].scaled(dtype="bf16", head_dim=64, n_q_heads=4, n_kv_heads=2, line_width=3, n_lines=12,
+                                     anchor_len=3, recent_lines=2, budget_lines=5)
+    assert w.mid_len == 6
+    for sn in ("mid", "cache"):
+        rep = run_parity(w.scaled(score_norm=sn))
+        _check(rep, w, allow_near_ties=1)
+        assert rep.compressions > 0
