@@ -155,6 +155,8 @@ def run_reference(args):
     if rank != 0:
         return
     w = W.WORKLOADS[args.workload]
+    if args.score_norm != "mid":
+        w = w.scaled(score_norm=args.score_norm)
     vals = []
     cb = None
     for i in range(args.warmup + args.steps):
@@ -399,6 +401,8 @@ def run_ours(args):
     w = W.WORKLOADS[args.workload]
     if args.layers:
         w = w.scaled(n_layers=args.layers)
+    if args.score_norm != "mid":
+        w = w.scaled(score_norm=args.score_norm)
 
     def bench_workload(wl, steps, warmup, sample_clocks, input_lines=0):
         r = Runner(wl, dev, args, input_lines=input_lines)
@@ -436,6 +440,7 @@ def run_ours(args):
                        "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
                        "storage": w.dtype, "prefix": w.cond_len, "grid": f"{w.n_lines}x{w.line_width}",
                        "budget_lines": w.budget_lines, "anchor": w.anchor_len, "recent_lines": w.recent_lines,
+                       "score_norm": w.score_norm,
                        "launch": ("cuda-graph per line, fused append+decode" + (", PDL" if not args.no_pdl else "") +
                                   (", line end per layer" if args.per_layer_line_end else ", one line-end launch for all layers")),
                        "l2": "inputs larger than L2: all layers cycled every token "
@@ -555,6 +560,8 @@ def main():
     ap.add_argument("--no-pdl", action="store_true")
     ap.add_argument("--per-layer-line-end", action="store_true", help="one line-end launch per layer instead of one for all layers")
     ap.add_argument("--tile-ranges", action="store_true", help="deal 32-row tiles, not whole units, to the decode CTAs")
+    ap.add_argument("--score-norm", default="mid", choices=["mid", "cache"],
+                    help="softmax of Eq. 9 over the mid keys (as written) or over the whole live cache (variant)")
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
