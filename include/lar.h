@@ -157,8 +157,16 @@ lar_status_t lar_decode_attn(lar_cache_t* c, int layer, const void* q, void* out
 lar_status_t lar_decode_step(lar_cache_t* c, int layer, const void* q, const void* k, const void* v,
                              void* out, void* stream);
 
-/* lar_decode_step with HOST buffers: copies q, k, v to a staging area of the slab, runs the fused
- * kernel and copies `out` back, all asynchronously on `stream` (use pinned memory). */
+/* lar_decode_step with HOST buffers (pinned memory): copies q, k, v to a staging area of the slab, runs the
+ * fused kernel and copies `out` back, asynchronously.  Seen from `stream` the call is one stream-ordered
+ * operation: `out_host` is complete once work enqueued on `stream` after the call runs (or `stream` is
+ * synchronised).  Inside, the copies run on two streams the cache owns and two staging slots alternate, so the
+ * copy-in of a call overlaps the kernel and copy-out of the call before it; the host buffers must stay
+ * untouched until then.  The call may be captured into a CUDA graph (the side streams join the capture and
+ * have re-joined `stream` when the call returns).
+ * k_host and v_host may both be NULL: q_host then holds q, k and v back to back in ONE host allocation (the
+ * layout a fused QKV projection leaves) and they cross the bus in one copy.  Adjacent but separately
+ * allocated buffers must be passed as three pointers. */
 lar_status_t lar_decode_step_host(lar_cache_t* c, int layer, const void* q_host, const void* k_host,
                                   const void* v_host, void* out_host, void* stream);
 

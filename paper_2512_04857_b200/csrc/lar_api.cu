@@ -4,6 +4,7 @@
 
 #include <cuda_runtime.h>
 #include <math.h>
+#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -26,6 +27,8 @@ thread_local int g_last_cuda_error = 0;
         if (e__ != cudaSuccess) {                        \
             g_last_cuda_error = (int)e__;                \
             (void)cudaGetLastError();                    \
+            if (getenv("LAR_DEBUG"))                     \
+                fprintf(stderr, "lar: line %d: %s -> %s\n", __LINE__, #call, cudaGetErrorString(e__)); \
             return LAR_ERR_CUDA;                         \
         }                                                \
     } while (0)
@@ -43,7 +46,8 @@ struct Layout {
     size_t off_scores, stride_scores;
     size_t off_kpool, off_vpool, stride_pool;
     size_t off_partials, off_tickets, tickets_bytes;  // decode scratch (shared by the layers)
-    size_t staging_q, staging_k, staging_v, staging_o;  // offsets inside the staging area
+    size_t staging_q, staging_k, staging_v, staging_o;  // offsets inside one staging slot
+    size_t staging_stride;                               // bytes between the two staging slots
     size_t total;
 };
 
@@ -156,7 +160,8 @@ void make_layout(const lar_config_t* c, const Derived& d, Layout& L) {
     L.staging_k = align_up(qb, 256);
     L.staging_v = L.staging_k + align_up(kb, 256);
     L.staging_o = L.staging_v + align_up(kb, 256);
-    L.off_staging = take(L.staging_o + qb);
+    L.staging_stride = align_up(L.staging_o + qb, 256);
+    L.off_staging = take(2 * L.staging_stride);
     L.stride_state = align_up(U * sizeof(lar::UnitState), 256);
     L.off_state = take(L.stride_state * Lyr);
     L.stride_ptab = align_up(U * d.ppu * 4, 256);
@@ -273,6 +278,24 @@ struct lar_cache {
     lar::TensorMaps tmaps;  // bf16 only
     int rows_per_layer;     // pool rows between consecutive layers
     std::vector<LayerShadow> sh;
+    // host-buffer entry point: copies run on streams of the library's own so that the inputs of the next call
+    // cross the bus while the kernel of this one runs
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t e_fork = nullptr, e_in[2] = {nullptr, nullptr}, e_k[2] = {nullptr, nullptr}, e_out = nullptr;
+    uint64_t host_calls = 0;
+    bool slot_used[2] = {false, false};
+    unsigned long long slot_capture[2] = {0, 0};  // capture the slot's kernel was recorded in (0: none, run eagerly)
+    unsigned long long last_host_capture = 0;
+    ~lar_cache() {
+        if (s_in) cudaStreamDestroy(s_in);
+        if (s_out) cudaStreamDestroy(s_out);
+        if (e_fork) cudaEventDestroy(e_fork);
+        if (e_out) cudaEventDestroy(e_out);
+        for (int i = 0; i < 2; ++i) {
+            if (e_in[i]) cudaEventDestroy(e_in[i]);
+            if (e_k[i]) cudaEventDestroy(e_k[i]);
+        }
+    }
 };
 
 namespace {
@@ -593,6 +616,14 @@ lar_status_t lar_cache_create(const lar_config_t* cfg, void* dev_slab, size_t sl
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, plan.decode_smem_bytes);
     if (ce == cudaSuccess && d.compressing)
         ce = cudaFuncSetAttribute((const void*)line_end_fn(*cfg, d.group), cudaFuncAttributeMaxDynamicSharedMemorySize, plan.line_end_smem_bytes);
+    if (ce == cudaSuccess) ce = cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking);
+    if (ce == cudaSuccess) ce = cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking);
+    if (ce == cudaSuccess) ce = cudaEventCreateWithFlags(&c->e_fork, cudaEventDisableTiming);
+    if (ce == cudaSuccess) ce = cudaEventCreateWithFlags(&c->e_out, cudaEventDisableTiming);
+    for (int i = 0; i < 2 && ce == cudaSuccess; ++i) {
+        ce = cudaEventCreateWithFlags(&c->e_in[i], cudaEventDisableTiming);
+        if (ce == cudaSuccess) ce = cudaEventCreateWithFlags(&c->e_k[i], cudaEventDisableTiming);
+    }
     if (ce == cudaSuccess) ce = cudaDeviceSynchronize();
     if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; (void)cudaGetLastError(); return fail(LAR_ERR_CUDA); }
     if (cfg->dtype == LAR_BF16) {
@@ -680,22 +711,69 @@ lar_status_t lar_decode_step(lar_cache_t* c, int layer, const void* q, const voi
     return LAR_OK;
 }
 
+// Host buffers in, host buffer out.  Three streams: the caller's (kernel), s_in (host -> device), s_out (device ->
+// host).  Two staging slots alternate, so the copy-in of call t + 1 overlaps the kernel and the copy-out of call t; the
+// caller's stream waits for the copy-out before the call returns its place in the stream, which keeps every effect of
+// the call ordered in that stream.  Works the same under stream capture: the side streams join the capture through
+// events and have re-joined the caller's stream when the call returns, so a capture may end after any call.
 lar_status_t lar_decode_step_host(lar_cache_t* c, int layer, const void* q_host, const void* k_host, const void* v_host,
                                   void* out_host, void* stream) {
-    if (bad_layer(c, layer) || !q_host || !k_host || !v_host || !out_host) return LAR_ERR_INVALID_ARG;
+    if (bad_layer(c, layer) || !q_host || !out_host || (!k_host) != (!v_host)) return LAR_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;
     const size_t qb = (size_t)c->cfg.batch * c->cfg.n_q_heads * c->d.row_bytes;
     const size_t kb = (size_t)c->cfg.batch * c->cfg.n_kv_heads * c->d.row_bytes;
-    char* stg = c->slab + c->L.off_staging;
-    LAR_CUDA(cudaMemcpyAsync(stg + c->L.staging_q, q_host, qb, cudaMemcpyHostToDevice, s));
-    LAR_CUDA(cudaMemcpyAsync(stg + c->L.staging_k, k_host, kb, cudaMemcpyHostToDevice, s));
-    LAR_CUDA(cudaMemcpyAsync(stg + c->L.staging_v, v_host, kb, cudaMemcpyHostToDevice, s));
+    const bool packed = !k_host;  // q | k | v back to back at q_host (one host allocation: one copy can span them)
+    if (packed) {
+        k_host = static_cast<const char*>(q_host) + qb;
+        v_host = static_cast<const char*>(q_host) + qb + kb;
+    }
+    const int slot = (int)(c->host_calls & 1u);
+    char* stg = c->slab + c->L.off_staging + c->L.staging_stride * slot;
+
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone, cap_in = cudaStreamCaptureStatusNone;
+    unsigned long long cap_id = 0, cap_in_id = 0;
+    LAR_CUDA(cudaStreamGetCaptureInfo(s, &cap, &cap_id));
+    LAR_CUDA(cudaStreamGetCaptureInfo(c->s_in, &cap_in, &cap_in_id));
+    const bool capturing = cap == cudaStreamCaptureStatusActive;
+    if (!capturing) cap_id = 0;
+    // When must s_in be ordered behind everything already in the caller's stream?  Under capture, if it is not part of
+    // the capture yet; eagerly, if the previous call was captured (its graph runs in the caller's stream).  Otherwise
+    // s_in only waits for the kernel that last read this staging slot.
+    const bool join = capturing ? cap_in != cudaStreamCaptureStatusActive : c->last_host_capture != 0;
+    if (join) {
+        LAR_CUDA(cudaEventRecord(c->e_fork, s));
+        LAR_CUDA(cudaStreamWaitEvent(c->s_in, c->e_fork, 0));
+    } else if (c->slot_used[slot] && c->slot_capture[slot] == cap_id) {
+        LAR_CUDA(cudaStreamWaitEvent(c->s_in, c->e_k[slot], 0));
+    }
+    // (a slot last used in an earlier capture or eagerly, seen from a new capture: that work precedes the graph in the
+    // caller's stream whenever the graph runs, and join is true for the capture's first call anyway)
+
+    if (packed && c->L.staging_k == qb && c->L.staging_v == qb + kb) {
+        LAR_CUDA(cudaMemcpyAsync(stg + c->L.staging_q, q_host, qb + 2 * kb, cudaMemcpyHostToDevice, c->s_in));  // q | k | v in one piece
+    } else {
+        LAR_CUDA(cudaMemcpyAsync(stg + c->L.staging_q, q_host, qb, cudaMemcpyHostToDevice, c->s_in));
+        LAR_CUDA(cudaMemcpyAsync(stg + c->L.staging_k, k_host, kb, cudaMemcpyHostToDevice, c->s_in));
+        LAR_CUDA(cudaMemcpyAsync(stg + c->L.staging_v, v_host, kb, cudaMemcpyHostToDevice, c->s_in));
+    }
+    LAR_CUDA(cudaEventRecord(c->e_in[slot], c->s_in));
+    LAR_CUDA(cudaStreamWaitEvent(s, c->e_in[slot], 0));
+
     const int saved = c->last_layer;
     c->last_layer = layer;  // a copy precedes the kernel: never prefetch ahead of it
     lar_status_t st = lar_decode_step(c, layer, stg + c->L.staging_q, stg + c->L.staging_k, stg + c->L.staging_v,
                                       stg + c->L.staging_o, stream);
-    if (st != LAR_OK) { c->last_layer = saved; return st; }
-    LAR_CUDA(cudaMemcpyAsync(out_host, stg + c->L.staging_o, qb, cudaMemcpyDeviceToHost, s));
+    if (st != LAR_OK) { c->last_layer = saved; return st; }   // s_in has re-joined the caller's stream above
+    LAR_CUDA(cudaEventRecord(c->e_k[slot], s));
+    c->slot_used[slot] = true;
+    c->slot_capture[slot] = cap_id;
+    c->last_host_capture = cap_id;
+    c->host_calls++;
+
+    LAR_CUDA(cudaStreamWaitEvent(c->s_out, c->e_k[slot], 0));
+    LAR_CUDA(cudaMemcpyAsync(out_host, stg + c->L.staging_o, qb, cudaMemcpyDeviceToHost, c->s_out));
+    LAR_CUDA(cudaEventRecord(c->e_out, c->s_out));
+    LAR_CUDA(cudaStreamWaitEvent(s, c->e_out, 0));
     return LAR_OK;
 }
 

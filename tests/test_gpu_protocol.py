@@ -121,6 +121,114 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     assert torch.equal(outs[0], outs[1])
 
 
+def _host_pipeline_inputs(cfg, steps, packed):
+    """Distinct pinned q, k, v per (step, layer); packed: q | k | v of a call adjacent in one buffer."""
+    L, S, Hq, Hkv, d = cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    g = torch.Generator(device="cpu").manual_seed(7)
+    nq, nk = S * Hq * d, S * Hkv * d
+    buf = torch.randn(steps, L, nq + 2 * nk, generator=g).to(torch.bfloat16).pin_memory()
+    if packed:
+        q, k, v = buf[..., :nq], buf[..., nq:nq + nk], buf[..., nq + nk:]
+    else:
+        q, k, v = (buf[..., :nq].contiguous().pin_memory(), buf[..., nq:nq + nk].contiguous().pin_memory(),
+                   buf[..., nq + nk:].contiguous().pin_memory())
+    return q, k, v
+
+
+def _device_path(cfg, b, q, k, v, steps):
+    """The same calls through the device-pointer entry point, synchronised after every call."""
+    L, S, Hq, Hkv, d, n = cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.line_width
+    c = lar.Cache(cfg)
+    for layer in range(L):
+        c.append_kv(layer, b["kc"], b["vc"], cfg.cond_len)
+    outs = torch.zeros(steps, L, S * Hq * d, dtype=torch.bfloat16)
+    for t in range(steps):
+        for layer in range(L):
+            c.decode_step(layer, q[t, layer].cuda().view(S, Hq, d), k[t, layer].cuda().view(S, Hkv, d),
+                          v[t, layer].cuda().view(S, Hkv, d), b["out"])
+            torch.cuda.synchronize()
+            outs[t, layer] = b["out"].cpu().view(-1)
+        if (t + 1) % n == 0:
+            for layer in range(L):
+                c.line_end_score_evict(layer)
+    assert c.poll_device_status() == 0
+    c.close()
+    return outs
+
+
+@pytest.mark.parametrize("packed", [False, True])
+def test_host_buffer_calls_back_to_back_without_synchronising(packed):
+    """The copies of consecutive calls overlap each other's kernels (two staging slots, library-owned copy streams):
+    distinct inputs per call, no synchronisation in between, line ends in the middle; results must be those of the
+    device-pointer entry point, bit for bit."""
+    cfg = _small(n_layers=3)
+    b = _bufs(cfg)
+    steps = 3 * cfg.line_width + 5
+    q, k, v = _host_pipeline_inputs(cfg, steps, packed)
+    ref = _device_path(cfg, b, q, k, v, steps)
+    c = lar.Cache(cfg)
+    for layer in range(cfg.n_layers):
+        c.append_kv(layer, b["kc"], b["vc"], cfg.cond_len)
+    outs = torch.zeros_like(ref).pin_memory()
+    for t in range(steps):
+        for layer in range(cfg.n_layers):
+            if packed:
+                c.decode_step_host(layer, q[t, layer], None, None, outs[t, layer])
+            else:
+                c.decode_step_host(layer, q[t, layer], k[t, layer], v[t, layer], outs[t, layer])
+        if (t + 1) % cfg.line_width == 0:
+            for layer in range(cfg.n_layers):
+                c.line_end_score_evict(layer)
+    torch.cuda.synchronize()
+    assert c.poll_device_status() == 0
+    c.close()
+    assert torch.equal(outs, ref)
+
+
+def test_host_buffer_calls_inside_cuda_graphs_then_eagerly():
+    """A line of host-buffer calls captured into a graph (the copy streams join the capture and re-join the capturing
+    stream by the end of every call), replayed line after line, followed by eager calls and a second capture."""
+    cfg = _small(n_layers=2, flags=lar.LAR_FLAG_NO_HOST_CHECKS)
+    b = _bufs(cfg)
+    n, L = cfg.line_width, cfg.n_layers
+    lines = 5
+    steps = lines * n
+    q, k, v = _host_pipeline_inputs(cfg, steps, True)
+    ref = _device_path(_small(n_layers=2), b, q, k, v, steps)
+    c = lar.Cache(cfg)
+    outs = torch.zeros_like(ref).pin_memory()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        for layer in range(L):
+            c.append_kv(layer, b["kc"], b["vc"], cfg.cond_len)
+
+        def line(t0):
+            for t in range(t0, t0 + n):
+                for layer in range(L):
+                    c.decode_step_host(layer, q[t, layer], None, None, outs[t, layer])
+            for layer in range(L):
+                c.line_end_score_evict(layer)
+
+        graphs = []
+        for ln in range(2):                       # lines 0 and 1: one graph each (different host addresses)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                line(ln * n)
+            graphs.append(g)
+        graphs[0].replay()
+        graphs[1].replay()
+        line(2 * n)                               # line 2 eagerly, right behind the graphs
+        g = torch.cuda.CUDAGraph()                # lines 3 and 4 in one more graph
+        with torch.cuda.graph(g, stream=s):
+            line(3 * n)
+            line(4 * n)
+        g.replay()
+    torch.cuda.synchronize()
+    assert c.poll_device_status() == 0
+    c.close()
+    assert torch.equal(outs, ref)
+
+
 def test_softmax_scale_override_and_single_row_cache():
     # C = 0 and the very first token: attention over one entry returns v exactly
     cfg = _small(n_layers=1, cond_len=0, softmax_scale=0.37, dtype="fp32")
