@@ -331,7 +331,7 @@ def measure_e2e(w, dev, args, steps=1):
     memory, runs the fused kernel and copies the output back (all inside the timed region)."""
     import torch
     from paper_2512_04857_b200 import lar, workloads as W
-    flags = lar.LAR_FLAG_NO_HOST_CHECKS
+    flags = lar.LAR_FLAG_NO_HOST_CHECKS | lar.LAR_FLAG_HOST_DEFER_OUT
     cfg = lar.config_from_workload(w, flags=flags, kv_splits=args.kv_splits, warps_per_cta=args.warps,
                                    stages=args.stages, page_tokens=args.page_tokens, decode_ctas=args.ctas)
     cache = lar.Cache(cfg, device=str(dev))
@@ -361,6 +361,7 @@ def measure_e2e(w, dev, args, steps=1):
                 if kind == "line+end":
                     for layer in range(L):
                         cache.line_end_score_evict(layer)     # (per layer here: the host copies of a layer precede its kernels)
+                cache.host_join()                             # the line's last copy-outs re-join the stream
             graphs.append(g)
 
         def gen():

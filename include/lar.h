@@ -73,6 +73,13 @@ typedef enum { LAR_BF16 = 0, LAR_FP32 = 1 } lar_dtype_t;
                                         the G heads.  The line-end kernel stages C + B keys in shared memory:
                                         configurations where they do not fit are rejected at creation. */
 
+#define LAR_FLAG_HOST_DEFER_OUT 0x20u /* lar_decode_step_host does not make `stream` wait for its copy-out: the
+                                        copy-out of a call then overlaps the kernels of the next calls as well.
+                                        `out_host` of a call is complete only after lar_cache_host_join (or four
+                                        further lar_decode_step_host calls) on the same stream.  Call
+                                        lar_cache_host_join before a stream capture ends and before switching
+                                        between captured and uncaptured calls (else LAR_ERR_BAD_STATE). */
+
 typedef struct lar_config {
     uint32_t struct_size;  /* = sizeof(lar_config_t) */
     int32_t n_layers;      /* L */
@@ -160,7 +167,7 @@ lar_status_t lar_decode_step(lar_cache_t* c, int layer, const void* q, const voi
 /* lar_decode_step with HOST buffers (pinned memory): copies q, k, v to a staging area of the slab, runs the
  * fused kernel and copies `out` back, asynchronously.  Seen from `stream` the call is one stream-ordered
  * operation: `out_host` is complete once work enqueued on `stream` after the call runs (or `stream` is
- * synchronised).  Inside, the copies run on two streams the cache owns and two staging slots alternate, so the
+ * synchronised).  Inside, the copies run on two streams the cache owns and four staging slots take turns, so the
  * copy-in of a call overlaps the kernel and copy-out of the call before it; the host buffers must stay
  * untouched until then.  The call may be captured into a CUDA graph (the side streams join the capture and
  * have re-joined `stream` when the call returns).
@@ -169,6 +176,10 @@ lar_status_t lar_decode_step(lar_cache_t* c, int layer, const void* q, const voi
  * allocated buffers must be passed as three pointers. */
 lar_status_t lar_decode_step_host(lar_cache_t* c, int layer, const void* q_host, const void* k_host,
                                   const void* v_host, void* out_host, void* stream);
+
+/* Makes `stream` wait for every copy-out that lar_decode_step_host deferred (LAR_FLAG_HOST_DEFER_OUT); a no-op
+ * otherwise.  No counterpart in the paper (host plumbing). */
+lar_status_t lar_cache_host_join(lar_cache_t* c, void* stream);
 
 /* Line-boundary step (Sec. 3.3, Eq. 5-10).  Legal only when the layer has just completed a line
  * (visual count multiple of n, every token decoded), else LAR_ERR_BAD_STATE.

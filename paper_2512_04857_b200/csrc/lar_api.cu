@@ -33,6 +33,8 @@ thread_local int g_last_cuda_error = 0;
         }                                                \
     } while (0)
 
+constexpr int kHostSlots = 4;  // staging slots of the host-buffer entry point (calls in flight)
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
@@ -47,7 +49,7 @@ struct Layout {
     size_t off_kpool, off_vpool, stride_pool;
     size_t off_partials, off_tickets, tickets_bytes;  // decode scratch (shared by the layers)
     size_t staging_q, staging_k, staging_v, staging_o;  // offsets inside one staging slot
-    size_t staging_stride;                               // bytes between the two staging slots
+    size_t staging_stride;                               // bytes between consecutive staging slots
     size_t total;
 };
 
@@ -161,7 +163,7 @@ void make_layout(const lar_config_t* c, const Derived& d, Layout& L) {
     L.staging_v = L.staging_k + align_up(kb, 256);
     L.staging_o = L.staging_v + align_up(kb, 256);
     L.staging_stride = align_up(L.staging_o + qb, 256);
-    L.off_staging = take(2 * L.staging_stride);
+    L.off_staging = take(kHostSlots * L.staging_stride);
     L.stride_state = align_up(U * sizeof(lar::UnitState), 256);
     L.off_state = take(L.stride_state * Lyr);
     L.stride_ptab = align_up(U * d.ppu * 4, 256);
@@ -281,17 +283,18 @@ struct lar_cache {
     // host-buffer entry point: copies run on streams of the library's own so that the inputs of the next call
     // cross the bus while the kernel of this one runs
     cudaStream_t s_in = nullptr, s_out = nullptr;
-    cudaEvent_t e_fork = nullptr, e_in[2] = {nullptr, nullptr}, e_k[2] = {nullptr, nullptr}, e_out = nullptr;
+    cudaEvent_t e_fork = nullptr, e_in[kHostSlots] = {}, e_k[kHostSlots] = {}, e_out[kHostSlots] = {};
+    bool out_pending[kHostSlots] = {};        // copy-out recorded in e_out[slot], not yet waited for by the caller's stream
     uint64_t host_calls = 0;
-    bool slot_used[2] = {false, false};
-    unsigned long long slot_capture[2] = {0, 0};  // capture the slot's kernel was recorded in (0: none, run eagerly)
+    bool slot_used[kHostSlots] = {};
+    unsigned long long slot_capture[kHostSlots] = {};  // capture the slot's kernel was recorded in (0: none, run eagerly)
     unsigned long long last_host_capture = 0;
     ~lar_cache() {
         if (s_in) cudaStreamDestroy(s_in);
         if (s_out) cudaStreamDestroy(s_out);
         if (e_fork) cudaEventDestroy(e_fork);
-        if (e_out) cudaEventDestroy(e_out);
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kHostSlots; ++i) {
+            if (e_out[i]) cudaEventDestroy(e_out[i]);
             if (e_in[i]) cudaEventDestroy(e_in[i]);
             if (e_k[i]) cudaEventDestroy(e_k[i]);
         }
@@ -619,8 +622,9 @@ lar_status_t lar_cache_create(const lar_config_t* cfg, void* dev_slab, size_t sl
     if (ce == cudaSuccess) ce = cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking);
     if (ce == cudaSuccess) ce = cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking);
     if (ce == cudaSuccess) ce = cudaEventCreateWithFlags(&c->e_fork, cudaEventDisableTiming);
-    if (ce == cudaSuccess) ce = cudaEventCreateWithFlags(&c->e_out, cudaEventDisableTiming);
-    for (int i = 0; i < 2 && ce == cudaSuccess; ++i) {
+    for (int i = 0; i < kHostSlots && ce == cudaSuccess; ++i) {
+        ce = cudaEventCreateWithFlags(&c->e_out[i], cudaEventDisableTiming);
+        if (ce != cudaSuccess) break;
         ce = cudaEventCreateWithFlags(&c->e_in[i], cudaEventDisableTiming);
         if (ce == cudaSuccess) ce = cudaEventCreateWithFlags(&c->e_k[i], cudaEventDisableTiming);
     }
@@ -712,7 +716,7 @@ lar_status_t lar_decode_step(lar_cache_t* c, int layer, const void* q, const voi
 }
 
 // Host buffers in, host buffer out.  Three streams: the caller's (kernel), s_in (host -> device), s_out (device ->
-// host).  Two staging slots alternate, so the copy-in of call t + 1 overlaps the kernel and the copy-out of call t; the
+// host).  kHostSlots staging slots take turns, so the copy-in of call t + 1 overlaps the kernel and the copy-out of call t; the
 // caller's stream waits for the copy-out before the call returns its place in the stream, which keeps every effect of
 // the call ordered in that stream.  Works the same under stream capture: the side streams join the capture through
 // events and have re-joined the caller's stream when the call returns, so a capture may end after any call.
@@ -727,7 +731,7 @@ lar_status_t lar_decode_step_host(lar_cache_t* c, int layer, const void* q_host,
         k_host = static_cast<const char*>(q_host) + qb;
         v_host = static_cast<const char*>(q_host) + qb + kb;
     }
-    const int slot = (int)(c->host_calls & 1u);
+    const int slot = (int)(c->host_calls % kHostSlots);
     char* stg = c->slab + c->L.off_staging + c->L.staging_stride * slot;
 
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone, cap_in = cudaStreamCaptureStatusNone;
@@ -736,6 +740,8 @@ lar_status_t lar_decode_step_host(lar_cache_t* c, int layer, const void* q_host,
     LAR_CUDA(cudaStreamGetCaptureInfo(c->s_in, &cap_in, &cap_in_id));
     const bool capturing = cap == cudaStreamCaptureStatusActive;
     if (!capturing) cap_id = 0;
+    for (int i = 0; i < kHostSlots; ++i)  // deferred copy-outs never cross a capture boundary: lar_cache_host_join comes first
+        if (c->out_pending[i] && c->slot_capture[i] != cap_id) return LAR_ERR_BAD_STATE;
     // When must s_in be ordered behind everything already in the caller's stream?  Under capture, if it is not part of
     // the capture yet; eagerly, if the previous call was captured (its graph runs in the caller's stream).  Otherwise
     // s_in only waits for the kernel that last read this staging slot.
@@ -758,6 +764,10 @@ lar_status_t lar_decode_step_host(lar_cache_t* c, int layer, const void* q_host,
     }
     LAR_CUDA(cudaEventRecord(c->e_in[slot], c->s_in));
     LAR_CUDA(cudaStreamWaitEvent(s, c->e_in[slot], 0));
+    if (c->out_pending[slot]) {  // deferred copy-out of kHostSlots calls ago: it reads the output slot this kernel writes
+        LAR_CUDA(cudaStreamWaitEvent(s, c->e_out[slot], 0));
+        c->out_pending[slot] = false;
+    }
 
     const int saved = c->last_layer;
     c->last_layer = layer;  // a copy precedes the kernel: never prefetch ahead of it
@@ -772,8 +782,27 @@ lar_status_t lar_decode_step_host(lar_cache_t* c, int layer, const void* q_host,
 
     LAR_CUDA(cudaStreamWaitEvent(c->s_out, c->e_k[slot], 0));
     LAR_CUDA(cudaMemcpyAsync(out_host, stg + c->L.staging_o, qb, cudaMemcpyDeviceToHost, c->s_out));
-    LAR_CUDA(cudaEventRecord(c->e_out, c->s_out));
-    LAR_CUDA(cudaStreamWaitEvent(s, c->e_out, 0));
+    LAR_CUDA(cudaEventRecord(c->e_out[slot], c->s_out));
+    if (c->cfg.flags & LAR_FLAG_HOST_DEFER_OUT)
+        c->out_pending[slot] = true;
+    else
+        LAR_CUDA(cudaStreamWaitEvent(s, c->e_out[slot], 0));
+    return LAR_OK;
+}
+
+lar_status_t lar_cache_host_join(lar_cache_t* c, void* stream) {
+    if (!c) return LAR_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    unsigned long long cap_id = 0;
+    LAR_CUDA(cudaStreamGetCaptureInfo(s, &cap, &cap_id));
+    if (cap != cudaStreamCaptureStatusActive) cap_id = 0;
+    for (int slot = 0; slot < kHostSlots; ++slot) {
+        if (!c->out_pending[slot]) continue;
+        if (c->slot_capture[slot] != cap_id) return LAR_ERR_BAD_STATE;  // recorded in another capture (or eagerly)
+        LAR_CUDA(cudaStreamWaitEvent(s, c->e_out[slot], 0));
+        c->out_pending[slot] = false;
+    }
     return LAR_OK;
 }
 

@@ -18,6 +18,7 @@ LAR_OK, LAR_ERR_INVALID_ARG, LAR_ERR_BAD_STATE, LAR_ERR_CAPACITY, LAR_ERR_CUDA, 
 LAR_BF16, LAR_FP32 = 0, 1
 LAR_FLAG_NO_HOST_CHECKS, LAR_FLAG_PDL, LAR_FLAG_SHUFFLE_PAGES, LAR_FLAG_TILE_RANGES = 0x1, 0x2, 0x4, 0x8
 LAR_FLAG_SCORE_CACHE_NORM = 0x10
+LAR_FLAG_HOST_DEFER_OUT = 0x20
 
 
 class lar_config_t(C.Structure):
@@ -68,6 +69,7 @@ def lib():
         "lar_decode_attn": (C.c_int, [vp, ip, vp, vp, vp]),
         "lar_decode_step": (C.c_int, [vp, ip, vp, vp, vp, vp, vp]),
         "lar_decode_step_host": (C.c_int, [vp, ip, vp, vp, vp, vp, vp]),
+        "lar_cache_host_join": (C.c_int, [vp, vp]),
         "lar_line_end_score_evict": (C.c_int, [vp, ip, vp]),
         "lar_line_end_score_evict_all": (C.c_int, [vp, vp]),
         "lar_cache_destroy": (C.c_int, [vp]),
@@ -162,6 +164,10 @@ def lar_decode_step(cache, layer, q, k, v, out, stream=None):
 def lar_decode_step_host(cache, layer, q, k, v, out, stream=None):
     _chk(lib().lar_decode_step_host(cache, layer, _ptr(q), _ptr(k), _ptr(v), _ptr(out), stream),
          "lar_decode_step_host")
+
+
+def lar_cache_host_join(cache, stream=None):
+    _chk(lib().lar_cache_host_join(cache, stream), "lar_cache_host_join")
 
 
 def lar_line_end_score_evict(cache, layer, stream=None):
@@ -260,6 +266,9 @@ class Cache:
 
     def decode_step_host(self, layer, q, k, v, out):
         lar_decode_step_host(self.handle, layer, q, k, v, out, self._stream())
+
+    def host_join(self):
+        lar_cache_host_join(self.handle, self._stream())
 
     def line_end_score_evict(self, layer):
         lar_line_end_score_evict(self.handle, layer, self._stream())

@@ -229,6 +229,53 @@ def test_host_buffer_calls_inside_cuda_graphs_then_eagerly():
     assert torch.equal(outs, ref)
 
 
+def test_host_buffer_calls_with_deferred_copy_out():
+    """LAR_FLAG_HOST_DEFER_OUT: the caller's stream does not wait for a call's copy-out until lar_cache_host_join (or
+    the second call after it).  Eager calls, then a graph per line with the join before the capture ends; a capture
+    that starts while copy-outs are pending is refused."""
+    cfg = _small(n_layers=2, flags=lar.LAR_FLAG_NO_HOST_CHECKS | lar.LAR_FLAG_HOST_DEFER_OUT)
+    b = _bufs(cfg)
+    n, L = cfg.line_width, cfg.n_layers
+    steps = 4 * n
+    q, k, v = _host_pipeline_inputs(cfg, steps, True)
+    ref = _device_path(_small(n_layers=2), b, q, k, v, steps)
+    c = lar.Cache(cfg)
+    outs = torch.zeros_like(ref).pin_memory()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        for layer in range(L):
+            c.append_kv(layer, b["kc"], b["vc"], cfg.cond_len)
+
+        def line(t0, join):
+            for t in range(t0, t0 + n):
+                for layer in range(L):
+                    c.decode_step_host(layer, q[t, layer], None, None, outs[t, layer])
+            for layer in range(L):
+                c.line_end_score_evict(layer)
+            if join:
+                c.host_join()
+
+        line(0, False)                            # eagerly; the last two copy-outs stay pending
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):       # pending copy-outs do not cross into a capture
+            st = _status(c.decode_step_host, 0, q[n, 0], None, None, outs[n, 0])
+        assert st == lar.LAR_ERR_BAD_STATE
+        c.host_join()
+        c.host_join()                             # nothing pending: no-op
+        graphs = []
+        for ln in range(1, 4):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                line(ln * n, True)
+            graphs.append(g)
+        for g in graphs:
+            g.replay()
+    torch.cuda.synchronize()
+    assert c.poll_device_status() == 0
+    c.close()
+    assert torch.equal(outs, ref)
+
+
 def test_softmax_scale_override_and_single_row_cache():
     # C = 0 and the very first token: attention over one entry returns v exactly
     cfg = _small(n_layers=1, cond_len=0, softmax_scale=0.37, dtype="fp32")
