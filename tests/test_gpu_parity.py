@@ -216,3 +216,15 @@ def test_bf16_mid_region_smaller_than_one_key_tile():
         rep = run_parity(w.scaled(score_norm=sn))
         _check(rep, w, allow_near_ties=1)
         assert rep.compressions > 0
+
+
+# ------------------------------------------------------------------ every layer of the deepest shapes
+@pytest.mark.parametrize("name", ["janus_pro_7b", "gqa_1024"])
+def test_every_layer_of_the_full_size_shape(name):
+    """All layers, full batch, whole generation in the benchmark's launch configuration (fused step, PDL, one
+    line-end launch for all layers); the oracle follows one unit of every layer (sequence and head vary with the layer)."""
+    w = W.WORKLOADS[name]
+    units = [(layer, (7 * layer + 3) % w.batch, (5 * layer + 1) % w.n_kv_heads) for layer in range(w.n_layers)]
+    rep = run_parity(w, units=units, gen_device="cuda", cfg_overrides=dict(flags=lar.LAR_FLAG_PDL), line_end_all=True)
+    _check(rep, w, allow_near_ties=3)
+    assert rep.compressions == w.n_layers * (w.n_lines - w.budget_lines)
