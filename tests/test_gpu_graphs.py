@@ -26,9 +26,9 @@ def _args(**kw):
     ("janus_pro_7b", dict(n_layers=3, batch=2, n_q_heads=4, n_kv_heads=4)),
     ("gqa_1024", dict(n_layers=2, batch=2, n_q_heads=8, n_kv_heads=2, n_lines=12)),
 ])
-@pytest.mark.parametrize("tile_ranges", [False, True])
-def test_graph_replay_of_a_second_generation_matches_the_oracle(shape, kw, tile_ranges):
-    w = W.WORKLOADS[shape].scaled(**kw)
+@pytest.mark.parametrize("tile_ranges,score_norm", [(False, "mid"), (True, "mid"), (False, "cache")])
+def test_graph_replay_of_a_second_generation_matches_the_oracle(shape, kw, tile_ranges, score_norm):
+    w = W.WORKLOADS[shape].scaled(score_norm=score_norm, **kw)
     dev = torch.device("cuda:0")
     r = bench.Runner(w, dev, _args(tile_ranges=tile_ranges))
     r.capture()
