@@ -484,7 +484,8 @@ def run_ours(args):
         line["e2e"] = {"value": world * w.images * w.n_visual / (float(em[0]) * 1e-3), "unit": UNIT,
                        "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"], "ms_per_step": float(em[0]),
                        "api": "lar_decode_step_host (pinned host q|k|v -> device, kernel, out -> host) per layer-step; "
-                              "copies on the library's own streams overlap the neighbouring calls' kernels"}
+                              "copies on the library's own streams overlap the neighbouring calls' kernels (deferred copy-out, "
+                              "joined once per line), one CUDA graph per line"}
     # ---- other benchmark shapes (not the headline line)
     if args.also:
         line["also"] = {}
