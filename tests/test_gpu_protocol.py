@@ -156,16 +156,17 @@ def _device_path(cfg, b, q, k, v, steps):
     return outs
 
 
-@pytest.mark.parametrize("packed", [False, True])
-def test_host_buffer_calls_back_to_back_without_synchronising(packed):
+@pytest.mark.parametrize("packed,flags", [(False, 0), (True, 0), (True, lar.LAR_FLAG_PDL),
+                                          (True, lar.LAR_FLAG_PDL | lar.LAR_FLAG_HOST_DEFER_OUT)])
+def test_host_buffer_calls_back_to_back_without_synchronising(packed, flags):
     """The copies of consecutive calls overlap each other's kernels (two staging slots, library-owned copy streams):
     distinct inputs per call, no synchronisation in between, line ends in the middle; results must be those of the
     device-pointer entry point, bit for bit."""
-    cfg = _small(n_layers=3)
+    cfg = _small(n_layers=3, flags=flags)
     b = _bufs(cfg)
     steps = 3 * cfg.line_width + 5
     q, k, v = _host_pipeline_inputs(cfg, steps, packed)
-    ref = _device_path(cfg, b, q, k, v, steps)
+    ref = _device_path(_small(n_layers=3), b, q, k, v, steps)
     c = lar.Cache(cfg)
     for layer in range(cfg.n_layers):
         c.append_kv(layer, b["kc"], b["vc"], cfg.cond_len)
@@ -179,6 +180,7 @@ def test_host_buffer_calls_back_to_back_without_synchronising(packed):
         if (t + 1) % cfg.line_width == 0:
             for layer in range(cfg.n_layers):
                 c.line_end_score_evict(layer)
+    c.host_join()                                   # (a no-op unless the copy-outs are deferred)
     torch.cuda.synchronize()
     assert c.poll_device_status() == 0
     c.close()
