@@ -124,3 +124,24 @@ def test_full_cache_budget_and_overrides():
     assert (p.warps_per_cta, p.stages, p.decode_ctas, p.page_tokens) == (3, 6, 40, 64)   # ring depth: multiple of 3 consumers and 2 producers
     # 4 units of up to 2 tiles (36 slots, 32-row tiles) dealt to 40 CTAs: every tile may sit in a CTA of its own
     assert p.max_segments == 2
+
+
+def test_cache_normalised_scoring_plan():
+    """LAR_FLAG_SCORE_CACHE_NORM stages C + B keys per unit in the line-end kernel: the plan's shared-memory figure
+    grows accordingly, every benchmark shape still fits, and a cache that cannot be staged is refused."""
+    for name, w in W.WORKLOADS.items():
+        base = lar.lar_plan_query(lar.config_from_workload(w))
+        var = lar.lar_plan_query(lar.config_from_workload(w.scaled(score_norm="cache")))
+        assert var.line_end_smem_bytes > base.line_end_smem_bytes, name
+        assert var.line_end_smem_bytes <= 227 * 1024, name
+        assert var.decode_smem_bytes == base.decode_smem_bytes and var.slab_bytes == base.slab_bytes
+        extra_rows = (w.cond_len + w.budget_tokens + 7) // 8 * 8 + 8 - (w.mid_len + 7) // 8 * 8
+        if w.dtype == "bf16":   # keys grow by extra_rows padded rows; the staged guide rows go away
+            nq16 = (w.line_width * w.group + 15) // 16 * 16
+            row = w.head_dim * 2 + 16
+            assert abs((var.line_end_smem_bytes - base.line_end_smem_bytes) - (extra_rows - nq16) * row) <= 16, name
+    big = W.WORKLOADS["gqa_1024"].scaled(score_norm="cache", cond_len=512)     # 1032 keys of 272 B > 227 KB
+    with pytest.raises(lar.LarError) as e:
+        lar.lar_plan_query(lar.config_from_workload(big))
+    assert e.value.status == lar.LAR_ERR_INVALID_ARG
+    lar.lar_plan_query(lar.config_from_workload(big.scaled(score_norm="mid")))  # the written form still fits
