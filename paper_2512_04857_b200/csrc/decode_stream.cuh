@@ -28,10 +28,11 @@
 //                    writes the output row (or the scratch partial + ticket), stores the new K/V
 //                    row, the index-map entry and the guide-queue row.
 // The producer never waits for arithmetic, so the HBM stream is continuous across unit boundaries.
-// Launched with programmatic dependent launch, the CTAs of the next layer's kernel move in as SMs free up
-// and wait for the preceding kernel in griddepcontrol.wait; where the host asks for it (prefetch = 1: two
-// CTAs fit per SM) the producer first fills its ring with tiles of this layer's cache, which the preceding
-// kernel (another layer) does not touch.
+// Launched with programmatic dependent launch, a CTA lets its dependents be scheduled at once and asks the
+// L2 to fetch every K/V tile of its range (a hint: L2 is the point of coherence, so a row that an earlier
+// kernel is still writing cannot be seen stale); only then does it wait for the preceding kernel in
+// griddepcontrol.wait.  With CTAs of at most half an SM, the kernels of the next layers are resident while
+// this one runs and HBM keeps streaming across launch boundaries; a kernel that starts finds its rows in L2.
 #pragma once
 #include <cuda.h>
 
@@ -59,8 +60,11 @@ struct StreamArgs {
     int len, n_tok;     // live rows per unit / visual tokens appended so far, before this step's append
     int unit_ranges;    // 1: CTA ranges end on unit boundaries
     int fused;          // 1: the step's token comes from k_new / v_new and is appended by this kernel
-    int prefetch;       // > 0: that many tiles of cached K/V per CTA may be fetched before the preceding kernel has finished
+    int prefetch;       // 1: the CTA may fill its ring before waiting for the preceding kernel (units whose length is published)
     int n_units, n_stages, max_seg;
+    int seq, need_seq;  // sequence number of this launch on its cache / of the launch that last wrote this layer's cache
+    int* done_seq;      // device word: every launch up to this number has completed
+    int q_slots, p_bufs;  // depth of the CTA's query ring / number of partial buffers
     int pool_row_base;  // first pool row of this layer in the tensor maps
 };
 
@@ -69,6 +73,10 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(dst),
         "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(policy)
         : "memory");
+}
+// hint: bring [p, p + bytes) into L2 (p 16-byte aligned, bytes a multiple of 16); no data reaches the SM
+__device__ __forceinline__ void l2_prefetch_bulk(const void* p, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
     uint64_t p;
@@ -97,6 +105,18 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&t);
 }
+// 2^x, x <= 0 or -inf (relative error 2^-22; -inf gives 0)
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// transpose of an 8 x 8 matrix of 16-bit elements held one 32-bit pair per thread (row lane / 4, columns 2 (lane % 4), + 1)
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
 
 template <int D>
@@ -120,17 +140,19 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {
 // ---- shared-memory plan of decode_stream_kernel (host and device agree through these) -------------
 constexpr int kMaxConsumers = 6;  // consumer warps per CTA at most
 constexpr int kProducers = 2;     // producer warps per CTA: tile j is fetched by producer j % kProducers
-__host__ __device__ constexpr int stream_q_slots(int G) { return G <= 2 ? 8 : 4; }
-__host__ __device__ constexpr int stream_partial_bufs(int) { return 2; }  // partial buffers per CTA
+constexpr int kMaxQSlots = 8;     // depth of the query ring at most
+// query ring / partial buffers of a CTA that works on at most `segs` segments per launch
+__host__ __device__ constexpr int stream_q_slots(int G, int segs) { const int q = G <= 2 ? 8 : 4; return segs < q ? (segs < 1 ? 1 : segs) : q; }
+__host__ __device__ constexpr int stream_partial_bufs(int segs) { return segs < 2 ? 1 : 2; }
 __host__ __device__ constexpr int stream_q_entry_bytes(int D, int G) { return ((G + 2) * D * 2 + 127) / 128 * 128; }
-__host__ __device__ constexpr int stream_fixed_smem_bytes(int D, int G, int W) {
-    return 1024                                               // slack: the ring starts on a 1024-byte boundary
-           + stream_q_slots(G) * stream_q_entry_bytes(D, G)   // query ring
-           + stream_partial_bufs(G) * (W + 1) * G * (D + 2) * 4  // partial buffers
-           + (2 * stream_q_slots(G) + 4) * 8 + 16;            // query / partial barriers, abort flag
+__host__ __device__ constexpr int stream_fixed_smem_bytes(int D, int G, int W, int NQ, int NPB) {
+    return 1024                                  // slack: the ring starts on a 1024-byte boundary
+           + NQ * stream_q_entry_bytes(D, G)     // query ring
+           + NPB * (W + 1) * G * (D + 2) * 4     // partial buffers
+           + (2 * kMaxQSlots + 4) * 8 + 16;      // query / partial barriers, abort flag
 }
-__host__ __device__ constexpr int stream_smem_bytes(int D, int G, int W, int NS) {
-    return stream_fixed_smem_bytes(D, G, W) + NS * (2 * (D / 64) * kStreamTile * 128 + 16);  // stage + its 2 barriers
+__host__ __device__ constexpr int stream_smem_bytes(int D, int G, int W, int NS, int NQ, int NPB) {
+    return stream_fixed_smem_bytes(D, G, W, NQ, NPB) + NS * (2 * (D / 64) * kStreamTile * 128 + 16);  // stage + its 2 barriers
 }
 
 // Wait on an mbarrier phase; gives up (and raises the CTA-wide abort flag) after ~1 s of SM clocks or as
@@ -153,31 +175,45 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
 // ---- optional in-kernel timeline (builds with -DLAR_TRACE only): per CTA 32 words; time stamps are
 // %globaltimer ns, waits are accumulated SM clocks of the recording warp's lane 0
 #ifdef LAR_TRACE
-__device__ unsigned long long lar_trace_buf[1024 * 32];
+__device__ unsigned long long lar_trace_buf[16 * 1024 * 32];
+#define LAR_TB (lar_trace_buf + (size_t)(a.seq & 15) * 1024 * 32)
 __device__ __forceinline__ unsigned long long trace_now() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-#define LAR_STAMP(slot) do { if ((threadIdx.x & 31) == 0) lar_trace_buf[blockIdx.x * 32 + (slot)] = trace_now(); } while (0)
+#define LAR_STAMP(slot) do { if ((threadIdx.x & 31) == 0) LAR_TB[blockIdx.x * 32 + (slot)] = trace_now(); } while (0)
 #ifdef LAR_TRACE_STAMPS_ONLY
 #define LAR_WAIT(slot, rec, call) (call)
 #else
 #define LAR_WAIT(slot, rec, call) [&]() { const long long t0__ = clock64(); const bool r__ = (call); \
-    if ((rec) && (threadIdx.x & 31) == 0) atomicAdd(&lar_trace_buf[blockIdx.x * 32 + (slot)], (unsigned long long)(clock64() - t0__)); return r__; }()
+    if ((rec) && (threadIdx.x & 31) == 0) atomicAdd(&LAR_TB[blockIdx.x * 32 + (slot)], (unsigned long long)(clock64() - t0__)); return r__; }()
 #endif
+#define LAR_ACC(slot, rec, val) do { if ((rec) && (threadIdx.x & 31) == 0) atomicAdd(&LAR_TB[blockIdx.x * 32 + (slot)], (unsigned long long)(val)); } while (0)
+#define LAR_CLK() clock64()
 #else
 #define LAR_STAMP(slot) do { } while (0)
 #define LAR_WAIT(slot, rec, call) (call)
+#define LAR_ACC(slot, rec, val) do { } while (0)
+#define LAR_CLK() 0ll
 #endif
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_gpu(int* p, int v) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ float exp2_or_zero(float m_part, float m_all) {
-    return m_part == -INFINITY ? 0.f : exp2f(m_part - m_all);
+    return m_part == -INFINITY ? 0.f : ex2_approx(m_part - m_all);
 }
 
 // A list of n items is dealt to P <= n CTAs in contiguous ranges, the first n % P of them one item longer.
@@ -197,8 +233,7 @@ template <int D, int G>
 __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs a, const __grid_constant__ TensorMaps tm) {
     using TR = MmaTraits<D>;
     using T16 = __nv_bfloat16;
-    constexpr int NQ = stream_q_slots(G);
-    constexpr int NPB = stream_partial_bufs(G);
+    const int NQ = a.q_slots, NPB = a.p_bufs;
     constexpr int QENT = stream_q_entry_bytes(D, G);
     constexpr int PS = D + 2;  // floats per (warp, head) partial: o[D], m, l
     constexpr int PER = D / 32;
@@ -219,9 +254,13 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     unsigned char* bars_ptr = reinterpret_cast<unsigned char*>(pbuf + NPB * pbuf_floats);
     const uint32_t bars = smem_u32(bars_ptr);
     const uint32_t bar_full = bars, bar_empty = bars + NS * 8;
-    const uint32_t bar_qfull = bars + 2 * NS * 8, bar_qempty = bar_qfull + NQ * 8;
-    const uint32_t bar_pfull = bar_qempty + NQ * 8, bar_pempty = bar_pfull + 2 * 8;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_ptr + (2 * NS + 2 * NQ + 4) * 8);
+    const uint32_t bar_qfull = bars + 2 * NS * 8, bar_qempty = bar_qfull + kMaxQSlots * 8;
+    const uint32_t bar_pfull = bar_qempty + kMaxQSlots * 8, bar_pempty = bar_pfull + 2 * 8;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_ptr + (2 * NS + 2 * kMaxQSlots + 4) * 8);
+
+    // Dependents may be scheduled from now on: they only hint the L2 before their own griddepcontrol.wait, and a
+    // dependent's wait covers this whole grid (which itself waits for its predecessor below).
+    grid_dep_launch();
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) {
@@ -242,7 +281,6 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     __syncthreads();
 
     if (threadIdx.x == 0) LAR_STAMP(0);
-    if (!a.prefetch) grid_dep_wait();
 
     // ---- the layer's tile list and this CTA's range of it
     const int len = a.len, n_tok = a.n_tok;
@@ -292,10 +330,17 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         // tiled copy per ~140 cycles, two keep the ring ahead of the consumers).  NS is a multiple of kProducers, so
         // a stage is always filled by the same producer.
         const int pw = warp;
-        bool dep_waited = !a.prefetch;
         bool ok = true;
-        const int fill_cap = a.prefetch < NS ? a.prefetch : NS;
-        const int fill_end = n_tiles < fill_cap ? n_tiles : fill_cap;
+        // ---- before the dependency: may the ring be filled already?  Every launch on a cache carries a sequence
+        // number; a decode kernel whose own dependency has resolved publishes the number of its predecessor (all
+        // launches up to that one have completed and their writes are visible to it).  The rows of this layer are
+        // final once the launch that last wrote them (need_seq, from the host) is covered by that word.
+        int fill_end = 0;
+        if (a.prefetch && ld_acquire_gpu(a.done_seq) >= a.need_seq) {
+            fence_proxy_async_global();  // the copies below read what the acquire made visible
+            fill_end = n_tiles < NS ? n_tiles : NS;
+        }
+        bool dep_waited = false;
         const int n_local = n_tiles > pw ? (n_tiles - pw + kProducers - 1) / kProducers : 0;
 
         auto describe = [&](int jj, int& y, int& rows, int& tile) {
@@ -335,12 +380,9 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             }
             const int cnt = n_local - i0 < 32 ? n_local - i0 : 32;
             for (int i = 0; i < cnt; ++i) {
-                const int j = kProducers * (i0 + i) + pw;
-                if (!dep_waited && j >= fill_end) {
-                    // the first tiles of this layer's cache are on their way; everything else depends on the preceding kernel
-                    grid_dep_wait();
-                    grid_dep_launch();
-                    LAR_STAMP(2);
+                if (!dep_waited && kProducers * (i0 + i) + pw >= fill_end) {
+                    grid_dep_wait();  // every tile from here on may still be written by the preceding kernels
+                    if (lane == 0) LAR_STAMP(2);
                     dep_waited = true;
                 }
                 const int yi = __shfl_sync(0xffffffffu, y, i), rti = __shfl_sync(0xffffffffu, rt, i);
@@ -366,16 +408,12 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                 }
             }
         }
-        if (!dep_waited) {
-            grid_dep_wait();
-            grid_dep_launch();
-        }
+        if (!dep_waited) grid_dep_wait();
         LAR_STAMP(3);
         if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
     } else if (warp < kProducers + W) {
         // =========================================================================== consumers
         grid_dep_wait();
-        grid_dep_launch();
         const int cw = warp - kProducers;
         const int quad = lane & 3, qrow = lane >> 2;  // fragment coordinates
         bool ok = true;
@@ -390,6 +428,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
 
             // ---- Q fragments (A operand): row qrow = head, 16 columns per k-step; heads >= G are zero rows
             const int qs = seg % NQ;
+            const long long tq0 = LAR_CLK();
             ok = LAR_WAIT(18, cw == 0, wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag));
             if (cw == 0 && seg == 0) LAR_STAMP(4);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
@@ -409,7 +448,9 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_qempty + qs * 8);
 
-            float m = -INFINITY, l = 0.f;  // head qrow; l is this thread's share of the row sum
+            LAR_ACC(27, cw == 0, LAR_CLK() - tq0);
+            // running maximum and this thread's share of the row sum of heads 2 quad and 2 quad + 1
+            float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
             // O^T: o[t][0], o[t][1] = heads 2 quad, 2 quad + 1 at d = 16 t + qrow; o[t][2], o[t][3] at d + 8
             float o[TR::KSTEPS][4];
 #pragma unroll
@@ -428,47 +469,59 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                 const int tile = t_begin + j - ub;
                 const int rows = len - tile * kStreamTile < kStreamTile ? len - tile * kStreamTile : kStreamTile;
                 const uint32_t St = ring + (uint32_t)s * TR::STAGE_BYTES;
+                const long long tc0 = LAR_CLK();
                 if (rows > 0) {
                     const int box_rows = (rows + 3) & ~3;  // K rows are lines 0.., V rows lines box_rows.. of a block
-                    // S[head][key] for the 32 keys of the tile: four n-tiles of 8 keys
-                    float sc[4][4];
+                    // S^T[key][head] = K q^T for the 32 keys of the tile: the keys are the M rows (two 16-key tiles), the
+                    // heads the 8 columns, so no MMA row is padding; even and odd k-steps go to accumulators of their own
+                    float c[2][2][4];
 #pragma unroll
-                    for (int jn = 0; jn < 4; ++jn) {
-                        sc[jn][0] = sc[jn][1] = sc[jn][2] = sc[jn][3] = 0.f;
+                    for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
-                        for (int i = 0; i < TR::KSTEPS / 2; ++i) {
-                            uint32_t b[4];
-                            ldmatrix_x4(St + tile_off<D>(8 * jn + (lane & 7), 4 * i + (lane >> 3)), b);
-                            mma_bf16(sc[jn], qa0[2 * i], 0u, qa2[2 * i], 0u, b[0], b[1]);
-                            mma_bf16(sc[jn], qa0[2 * i + 1], 0u, qa2[2 * i + 1], 0u, b[2], b[3]);
+                        for (int e = 0; e < 2; ++e) c[mt][e][0] = c[mt][e][1] = c[mt][e][2] = c[mt][e][3] = 0.f;
+#pragma unroll
+                        for (int ks = 0; ks < TR::KSTEPS; ++ks) {
+                            uint32_t af[4];  // keys 16 mt + (lane & 15), 16 dims from 16 ks
+                            ldmatrix_x4(St + tile_off<D>(16 * mt + (lane & 15), 2 * ks + (lane >> 4)), af);
+                            mma_bf16(c[mt][ks & 1], af[0], af[1], af[2], af[3], qa0[ks], qa2[ks]);
                         }
                     }
-                    // online softmax over the keys this thread holds: 8 jn + 2 quad, + 1
-                    float sv[8];
+                    // this thread: keys qrow + {0, 8, 16, 24}, heads 2 quad and 2 quad + 1
+                    float sv[4][2];
 #pragma unroll
-                    for (int jn = 0; jn < 4; ++jn) {
-                        sv[2 * jn + 0] = (8 * jn + 2 * quad + 0 < rows) ? sc[jn][0] * a.scale_log2 : -INFINITY;
-                        sv[2 * jn + 1] = (8 * jn + 2 * quad + 1 < rows) ? sc[jn][1] * a.scale_log2 : -INFINITY;
+                    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                        for (int hf = 0; hf < 2; ++hf) {
+                            const bool live = 16 * mt + 8 * hf + qrow < rows;
+                            sv[2 * mt + hf][0] = live ? (c[mt][0][2 * hf] + c[mt][1][2 * hf]) * a.scale_log2 : -INFINITY;
+                            sv[2 * mt + hf][1] = live ? (c[mt][0][2 * hf + 1] + c[mt][1][2 * hf + 1]) * a.scale_log2 : -INFINITY;
+                        }
+                    float mx0 = fmaxf(fmaxf(sv[0][0], sv[1][0]), fmaxf(sv[2][0], sv[3][0]));
+                    float mx1 = fmaxf(fmaxf(sv[0][1], sv[1][1]), fmaxf(sv[2][1], sv[3][1]));
+#pragma unroll
+                    for (int off = 4; off <= 16; off <<= 1) {
+                        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
                     }
-                    float mx = fmaxf(fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3])), fmaxf(fmaxf(sv[4], sv[5]), fmaxf(sv[6], sv[7])));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                    const float m_new = fmaxf(m, mx);
-                    const float corr = exp2f(m - m_new);
-                    float pr[8];
+                    // rows >= 1: the tile has a live key, so the new maxima are finite
+                    const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+                    const float ca = ex2_approx(m0 - mn0), cb = ex2_approx(m1 - mn1);
+                    float pr[4][2];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) pr[i] = exp2f(sv[i] - m_new);
-                    l = l * corr + ((pr[0] + pr[1]) + (pr[2] + pr[3])) + ((pr[4] + pr[5]) + (pr[6] + pr[7]));
-                    m = m_new;
-                    if (__any_sync(0xffffffffu, corr != 1.f)) {
-                        // the accumulator columns of this thread belong to heads 2 quad and 2 quad + 1
-                        const float ca = __shfl_sync(0xffffffffu, corr, 8 * quad), cb = __shfl_sync(0xffffffffu, corr, 8 * quad + 4);
-#pragma unroll
-                        for (int t = 0; t < TR::KSTEPS; ++t) { o[t][0] *= ca; o[t][1] *= cb; o[t][2] *= ca; o[t][3] *= cb; }
+                    for (int k = 0; k < 4; ++k) {
+                        pr[k][0] = ex2_approx(sv[k][0] - mn0);
+                        pr[k][1] = ex2_approx(sv[k][1] - mn1);
                     }
-                    // P^T as B operand: keys 0-15 and keys 16-31
-                    const uint32_t pb00 = pack_bf16(pr[0], pr[1]), pb01 = pack_bf16(pr[2], pr[3]);
-                    const uint32_t pb10 = pack_bf16(pr[4], pr[5]), pb11 = pack_bf16(pr[6], pr[7]);
+                    l0 = l0 * ca + ((pr[0][0] + pr[1][0]) + (pr[2][0] + pr[3][0]));
+                    l1 = l1 * cb + ((pr[0][1] + pr[1][1]) + (pr[2][1] + pr[3][1]));
+                    m0 = mn0;
+                    m1 = mn1;
+                    // the accumulator columns of this thread belong to the same two heads
+#pragma unroll
+                    for (int t = 0; t < TR::KSTEPS; ++t) { o[t][0] *= ca; o[t][1] *= cb; o[t][2] *= ca; o[t][3] *= cb; }
+                    // P^T as B operand (keys 2 quad, 2 quad + 1 of an 8-key block; head qrow): transpose the 8 x 8 blocks
+                    const uint32_t pb00 = movmatrix_trans(pack_bf16(pr[0][0], pr[0][1])), pb01 = movmatrix_trans(pack_bf16(pr[1][0], pr[1][1]));
+                    const uint32_t pb10 = movmatrix_trans(pack_bf16(pr[2][0], pr[2][1])), pb11 = movmatrix_trans(pack_bf16(pr[3][0], pr[3][1]));
                     // a short box leaves the lines behind its V rows unwritten: their weight is 0, but
                     // 0 * (stale NaN) is not
                     if (box_rows < kStreamTile) {
@@ -492,8 +545,11 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_empty + s * 8);
+                LAR_ACC(23, cw == 0, LAR_CLK() - tc0);
+                LAR_ACC(24, cw == 0, 1);
             }
             if (!ok) break;
+            const long long ts0 = LAR_CLK();
 
             // ---- this warp's partial of the segment -> shared memory
             const int buf = seg % NPB;
@@ -501,8 +557,11 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                 ok = LAR_WAIT(20, cw == 0, wait_or_abort(bar_pempty + buf * 8, (uint32_t)((seg / NPB - 1) & 1), abort_flag));
                 if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             }
-            l += __shfl_xor_sync(0xffffffffu, l, 1);
-            l += __shfl_xor_sync(0xffffffffu, l, 2);
+#pragma unroll
+            for (int off = 4; off <= 16; off <<= 1) {
+                l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+                l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+            }
             {
                 float* wp = pbuf + buf * pbuf_floats + cw * G * PS;
                 if (2 * quad < G) {
@@ -511,6 +570,10 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                         wp[2 * quad * PS + 16 * t + qrow] = o[t][0];
                         wp[2 * quad * PS + 16 * t + 8 + qrow] = o[t][2];
                     }
+                    if (qrow == 0) {
+                        wp[2 * quad * PS + D] = m0;
+                        wp[2 * quad * PS + D + 1] = l0;
+                    }
                 }
                 if (2 * quad + 1 < G) {
 #pragma unroll
@@ -518,21 +581,23 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                         wp[(2 * quad + 1) * PS + 16 * t + qrow] = o[t][1];
                         wp[(2 * quad + 1) * PS + 16 * t + 8 + qrow] = o[t][3];
                     }
-                }
-                if (qrow < G && quad == 0) {
-                    wp[qrow * PS + D] = m;
-                    wp[qrow * PS + D + 1] = l;
+                    if (qrow == 0) {
+                        wp[(2 * quad + 1) * PS + D] = m1;
+                        wp[(2 * quad + 1) * PS + D + 1] = l1;
+                    }
                 }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_pfull + buf * 8);
+            LAR_ACC(25, cw == 0, LAR_CLK() - ts0);
+            LAR_ACC(26, cw == 0, 1);
         }
         if (cw == 0) LAR_STAMP(6);
         if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
     } else {
         // =========================================================================== epilogue
         grid_dep_wait();
-        grid_dep_launch();
+        if (p == 0 && lane == 0) st_release_gpu(a.done_seq, a.seq - 1);  // everything before this launch has completed
         bool ok = true;
         if (lane == 0)
             for (int sg = 0; sg < NQ && sg < n_segs && ok; ++sg) ok = issue_inputs(sg);  // the input ring's first round

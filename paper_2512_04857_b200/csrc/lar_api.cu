@@ -57,6 +57,7 @@ struct Derived {
     int units, group, elt, row_bytes, cap, ppu, P, cap_pad, M, mid_pad, compressing, B, N;
     int ctas, max_seg;  // bf16 decode: CTAs of the persistent grid, most segments one unit is cut into
     int unit_ranges;    // bf16 decode: 1 if the CTAs' ranges end on unit boundaries
+    int q_slots, p_bufs;  // bf16 decode: depth of a CTA's query ring, number of its partial buffers
     int le_threads;     // threads per CTA of the line-end kernel
 };
 
@@ -132,6 +133,13 @@ bool derive(const lar_config_t* c, Derived& d) {
         d.unit_ranges = (d.units >= d.ctas && (long long)d.units * 10 >= per * d.ctas * 8) ? 1 : 0;
         if (c->flags & LAR_FLAG_TILE_RANGES) d.unit_ranges = 0;
     }
+    {
+        // segments a CTA works on per launch at most: whole units, or (tile ranges) not known in closed form
+        const int pe = d.units < d.ctas ? d.units : d.ctas;
+        const int segs = d.unit_ranges ? (d.units + pe - 1) / pe : 8;
+        d.q_slots = lar::stream_q_slots(d.group, segs);
+        d.p_bufs = lar::stream_partial_bufs(segs);
+    }
     // A unit of T tiles is cut into at most ceil(T / floor(U T / P)) + 1 segments (never more than T or P).
     // line end: one CTA per unit, 8 warps; few units with a large mid region get one warp per 16 guide rows (16..32 warps)
     d.le_threads = 256;
@@ -206,7 +214,7 @@ void choose_plan(const lar_config_t* c, const Derived& d, lar_plan_t& p) {
         p.stages = NS;
         p.decode_ctas = d.ctas;
         p.max_segments = d.max_seg;
-        p.decode_smem_bytes = c->head_dim == 64 ? lar::stream_smem_bytes(64, d.group, W, NS) : lar::stream_smem_bytes(128, d.group, W, NS);
+        p.decode_smem_bytes = lar::stream_smem_bytes(c->head_dim, d.group, W, NS, d.q_slots, d.p_bufs);
         return;
     }
     const int tiles = (d.cap + lar::kGranule - 1) / lar::kGranule;  // tiles at the longest live length
@@ -277,6 +285,8 @@ struct lar_cache {
     float scale;
     uint64_t launches;
     int last_layer;  // layer whose cache the most recent library kernel may have written (-1 none)
+    int seq;         // launches on this cache since the last reset (the kernels that write a cache are numbered)
+    std::vector<int> last_writer;  // per layer: number of the launch that last wrote the layer's cache (0: none)
     lar::TensorMaps tmaps;  // bf16 only
     int rows_per_layer;     // pool rows between consecutive layers
     std::vector<LayerShadow> sh;
@@ -429,6 +439,7 @@ lar_status_t launch_append(lar_cache* c, int layer, const void* k, const void* v
     LAR_CUDA(cudaGetLastError());
     c->launches++;
     c->last_layer = layer;
+    c->last_writer[layer] = ++c->seq;
     return LAR_OK;
 }
 
@@ -439,7 +450,10 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
     // preceding kernel is done.  It requests its first ring of cached K/V tiles then, so that arithmetic starts when
     // the dependency resolves.
     int prefetch = 0;
-    if (pdl && c->last_layer != layer && c->last_layer >= 0) prefetch = c->cfg.dtype == LAR_BF16 ? c->plan.stages : 1;
+    if (c->cfg.dtype == LAR_BF16)
+        prefetch = pdl ? 1 : 0;
+    else if (pdl && c->last_layer != layer && c->last_layer >= 0)
+        prefetch = 1;
     const float scale_log2 = c->scale * 1.4426950408889634f;
 
     cudaLaunchConfig_t lc;
@@ -481,6 +495,12 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
         a.n_units = c->d.units;
         a.n_stages = c->plan.stages;
         a.max_seg = c->d.max_seg;
+        a.seq = ++c->seq;
+        a.need_seq = c->last_writer[layer];
+        c->last_writer[layer] = a.seq;
+        a.done_seq = reinterpret_cast<int*>(c->slab + c->L.off_status + 128);
+        a.q_slots = c->d.q_slots;
+        a.p_bufs = c->d.p_bufs;
         a.pool_row_base = layer * c->rows_per_layer;
         lc.gridDim = dim3((unsigned)c->d.ctas, 1, 1);
         lc.blockDim = dim3((unsigned)(32 * (c->plan.warps_per_cta + lar::kProducers + 1)), 1, 1);
@@ -584,6 +604,8 @@ lar_status_t lar_cache_create(const lar_config_t* cfg, void* dev_slab, size_t sl
     c->launches = 0;
     c->last_layer = -1;
     c->sh.assign((size_t)cfg->n_layers, LayerShadow());
+    c->seq = 0;
+    c->last_writer.assign((size_t)cfg->n_layers, 0);
 
     auto fail = [&](lar_status_t e) { delete c; return e; };
     cudaError_t ce = cudaGetDevice(&c->device);
@@ -648,8 +670,11 @@ lar_status_t lar_cache_reset(lar_cache_t* c, void* stream) {
     if (!c) return LAR_ERR_INVALID_ARG;
     LAR_CUDA(cudaMemsetAsync(c->slab + c->L.off_state, 0, c->L.stride_state * c->cfg.n_layers, (cudaStream_t)stream));
     LAR_CUDA(cudaMemsetAsync(c->slab + c->L.off_tickets, 0, c->L.tickets_bytes, (cudaStream_t)stream));
+    LAR_CUDA(cudaMemsetAsync(c->slab + c->L.off_status + 128, 0, sizeof(int), (cudaStream_t)stream));
     for (auto& s : c->sh) s = LayerShadow();
     c->last_layer = -1;
+    c->seq = 0;
+    c->last_writer.assign(c->last_writer.size(), 0);
     return LAR_OK;
 }
 
@@ -831,6 +856,7 @@ lar_status_t lar_line_end_score_evict(lar_cache_t* c, int layer, void* stream) {
         LAR_CUDA(cudaGetLastError());
         c->launches++;
         c->last_layer = layer;
+        c->last_writer[layer] = ++c->seq;
         if (sh.v >= c->d.B) sh.v -= c->cfg.line_width;
     }
     sh.line_fill = 0;
@@ -851,6 +877,7 @@ lar_status_t lar_line_end_score_evict_all(lar_cache_t* c, void* stream) {
         LAR_CUDA(cudaGetLastError());
         c->launches++;
         c->last_layer = -2;  // every layer's cache was just written: the next decode launch must not fetch ahead
+        c->last_writer.assign(c->last_writer.size(), ++c->seq);
         for (LayerShadow& sh : c->sh)
             if (sh.v >= c->d.B) sh.v -= c->cfg.line_width;
     }
@@ -889,10 +916,10 @@ lar_status_t lar_cache_get_state(lar_cache_t* c, int layer, int32_t* lens, int32
 #ifdef LAR_TRACE
 // Trace builds only: copy the in-kernel timeline of the decode kernel (32 words per CTA) to the host and clear it.
 lar_status_t lar_debug_trace_read(unsigned long long* host_out, int n_ctas) {
-    if (!host_out || n_ctas < 1 || n_ctas > 1024) return LAR_ERR_INVALID_ARG;
+    if (!host_out || n_ctas != 1024) return LAR_ERR_INVALID_ARG;
     LAR_CUDA(cudaDeviceSynchronize());
-    LAR_CUDA(cudaMemcpyFromSymbol(host_out, lar::lar_trace_buf, sizeof(unsigned long long) * 32 * (size_t)n_ctas));
-    static unsigned long long zeros[1024 * 32];
+    LAR_CUDA(cudaMemcpyFromSymbol(host_out, lar::lar_trace_buf, sizeof(unsigned long long) * 32 * 16 * (size_t)n_ctas));
+    static unsigned long long zeros[16 * 1024 * 32];
     LAR_CUDA(cudaMemcpyToSymbol(lar::lar_trace_buf, zeros, sizeof(zeros)));
     return LAR_OK;
 }

@@ -15,8 +15,9 @@ __global__ void __launch_bounds__(128) append_kernel(const LayerView lv, const T
                                                      const T* __restrict__ v, int n_tokens, int is_prefix) {
     constexpr int ROW_BYTES = D * (int)sizeof(T);
     constexpr int CHUNKS = ROW_BYTES / 16;
+    // No early release of dependents: a decode kernel launched behind this one may read the cache as soon as it is
+    // scheduled, so it must not be scheduled before this grid has completed.
     grid_dep_wait();
-    grid_dep_launch();
     const int unit = blockIdx.x;
     const UnitState st = lv.state[unit];
     const int room = lv.cap - st.len;
@@ -175,8 +176,8 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
     constexpr int CHUNKS = ROW_BYTES / 16;
     constexpr int KROW = ROW_BYTES + 16;
     extern __shared__ __align__(128) unsigned char smem[];
+    // (no early release of dependents, as in append_kernel: rows move until the very end)
     grid_dep_wait();
-    grid_dep_launch();
 
     const LayerView lv = layer_view_at(lv0, ls, (int)blockIdx.y);
     const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, W = blockDim.x >> 5;
