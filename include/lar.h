@@ -55,13 +55,15 @@ typedef enum { LAR_BF16 = 0, LAR_FP32 = 1 } lar_dtype_t;
                                         generation in order and replay the graphs in that same order (the
                                         kernels check the length against device memory and record bit 16
                                         otherwise).  Device-side checks stay active. */
-#define LAR_FLAG_PDL 0x2u            /* launch decode kernels with programmatic dependent launch and
-                                        let them prefetch cached K/V before the preceding kernel on the
-                                        stream has finished.  Contract: the kernel enqueued on `stream`
-                                        immediately before a decode call of layer l does not write layer
-                                        l's cache (the library checks this for its own launches), and any
-                                        caller kernel using PDL waits on its own dependency before it
-                                        triggers its dependents. */
+#define LAR_FLAG_PDL 0x2u            /* launch decode kernels with programmatic dependent launch: a decode kernel lets
+                                        its successors be scheduled at once, and a successor may fetch cached K/V of
+                                        its own layer before the preceding kernels on the stream have finished.  The
+                                        library guards this itself: launches on a cache are numbered, a device word
+                                        records up to which number they have completed, and a kernel fetches ahead
+                                        only if the launch that last wrote its layer's cache is covered.  Contract
+                                        for the caller: a kernel of its own that uses programmatic dependent launch
+                                        on the same stream waits on its dependency before it completes, and nothing
+                                        but this library writes the slab. */
 #define LAR_FLAG_SHUFFLE_PAGES 0x4u  /* test hook: assign physical pages in a pseudo-random order */
 #define LAR_FLAG_TILE_RANGES 0x8u    /* bf16 decode: always deal 32-row tiles (not whole units) to the CTAs, even
                                         where whole units would balance well enough */

@@ -9,27 +9,18 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "liblar.so")
-OUT_TRACE = os.path.join(HERE, "liblar_trace.so")
 SOURCES = [os.path.join(CSRC, "lar_api.cu")]
 DEPS = SOURCES + [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cuh")] + \
     [os.path.join(ROOT, "include", "lar.h")]
 
 
-def nvcc_cmd(verbose: bool = False, trace: bool = False):
+def nvcc_cmd(verbose: bool = False):
     cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xcompiler", "-fPIC", "-shared",
-           "-I", os.path.join(ROOT, "include"), "-o", OUT_TRACE if trace else OUT] + SOURCES
-    if trace:
-        cmd[1:1] = ["-DLAR_TRACE"] + (["-DLAR_TRACE_STAMPS_ONLY"] if os.environ.get("LAR_TRACE_STAMPS_ONLY") else [])
+           "-I", os.path.join(ROOT, "include"), "-o", OUT] + SOURCES
     if verbose:
         cmd[1:1] = ["-Xptxas", "-v"]
     return cmd
-
-
-def build_trace() -> str:
-    """Diagnostic build with the decode kernel's in-kernel timeline compiled in (liblar_trace.so)."""
-    subprocess.run(nvcc_cmd(trace=True), check=True)
-    return OUT_TRACE
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -40,7 +31,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    if "--trace" in sys.argv:
-        print(build_trace())
-    else:
-        print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv))

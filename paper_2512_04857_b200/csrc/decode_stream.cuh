@@ -17,22 +17,22 @@
 //   warps 0, 1       producers: walk the CTA's tile range (every other tile each) and keep a ring of NS
 //                    stages filled with K and V tiles (cp.async.bulk.tensor, 3-D tiled, 128-byte swizzle).
 //   next W warps     consumers: tile j of the range goes to consumer j % W:
-//                        S = Q K^T     mma.sync m16n8k16 (bf16 in, fp32 out), rows = the G heads
-//                        online softmax in fp32 (base-2, scale folded into the logits)
-//                        O^T += V^T P^T  same instruction with the d rows as M: the logits' accumulator
-//                                      layout is the B-operand layout of P^T, V^T fragments come from
-//                                      ldmatrix.trans, and no accumulator row is wasted on padding
+//                        S^T = K q^T   mma.sync m16n8k16 (bf16 in, fp32 out): the 32 keys of the tile are the M rows,
+//                                      the G heads the 8 columns, so no MMA row is padding
+//                        online softmax in fp32 (base-2 ex2.approx, scale folded into the logits)
+//                        O^T += V^T P^T  same instruction with the d rows as M: P^T (B operand) is the 8 x 8
+//                                      transposes (movmatrix) of the packed probabilities, V^T fragments come from
+//                                      ldmatrix.trans
 //                    and at the end of a segment each consumer leaves its partial in shared memory.
 //   last warp        epilogue: fetches the queries (and the step's new k, v row) of each segment into a
 //                    small ring; merges the W partials of a segment with the step's own token,
 //                    writes the output row (or the scratch partial + ticket), stores the new K/V
 //                    row, the index-map entry and the guide-queue row.
 // The producer never waits for arithmetic, so the HBM stream is continuous across unit boundaries.
-// Launched with programmatic dependent launch, a CTA lets its dependents be scheduled at once and asks the
-// L2 to fetch every K/V tile of its range (a hint: L2 is the point of coherence, so a row that an earlier
-// kernel is still writing cannot be seen stale); only then does it wait for the preceding kernel in
-// griddepcontrol.wait.  With CTAs of at most half an SM, the kernels of the next layers are resident while
-// this one runs and HBM keeps streaming across launch boundaries; a kernel that starts finds its rows in L2.
+// Launched with programmatic dependent launch, a CTA lets its dependents be scheduled at once; the CTAs of the next
+// layers' kernels move in as SMs free up and, before their own griddepcontrol.wait, fill their rings with tiles of
+// their layer's cache -- if the cache's completion word shows that the launch that last wrote that layer has
+// completed (every decode kernel publishes, after its own wait, the sequence number of its predecessor).
 #pragma once
 #include <cuda.h>
 
@@ -172,32 +172,6 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
     }
     return true;
 }
-// ---- optional in-kernel timeline (builds with -DLAR_TRACE only): per CTA 32 words; time stamps are
-// %globaltimer ns, waits are accumulated SM clocks of the recording warp's lane 0
-#ifdef LAR_TRACE
-__device__ unsigned long long lar_trace_buf[16 * 1024 * 32];
-#define LAR_TB (lar_trace_buf + (size_t)(a.seq & 15) * 1024 * 32)
-__device__ __forceinline__ unsigned long long trace_now() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-#define LAR_STAMP(slot) do { if ((threadIdx.x & 31) == 0) LAR_TB[blockIdx.x * 32 + (slot)] = trace_now(); } while (0)
-#ifdef LAR_TRACE_STAMPS_ONLY
-#define LAR_WAIT(slot, rec, call) (call)
-#else
-#define LAR_WAIT(slot, rec, call) [&]() { const long long t0__ = clock64(); const bool r__ = (call); \
-    if ((rec) && (threadIdx.x & 31) == 0) atomicAdd(&LAR_TB[blockIdx.x * 32 + (slot)], (unsigned long long)(clock64() - t0__)); return r__; }()
-#endif
-#define LAR_ACC(slot, rec, val) do { if ((rec) && (threadIdx.x & 31) == 0) atomicAdd(&LAR_TB[blockIdx.x * 32 + (slot)], (unsigned long long)(val)); } while (0)
-#define LAR_CLK() clock64()
-#else
-#define LAR_STAMP(slot) do { } while (0)
-#define LAR_WAIT(slot, rec, call) (call)
-#define LAR_ACC(slot, rec, val) do { } while (0)
-#define LAR_CLK() 0ll
-#endif
-
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -280,7 +254,6 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     }
     __syncthreads();
 
-    if (threadIdx.x == 0) LAR_STAMP(0);
 
     // ---- the layer's tile list and this CTA's range of it
     const int len = a.len, n_tok = a.n_tok;
@@ -310,7 +283,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     // producer's first K/V copies are not queued behind them.
     auto issue_inputs = [&](int seg) -> bool {
         const int slot = seg % NQ;
-        if (seg >= NQ && !LAR_WAIT(17, true, wait_or_abort(bar_qempty + slot * 8, (uint32_t)((seg / NQ - 1) & 1), abort_flag))) return false;
+        if (seg >= NQ && !wait_or_abort(bar_qempty + slot * 8, (uint32_t)((seg / NQ - 1) & 1), abort_flag)) return false;
         const int unit = u0 + seg;
         const bool closes = (unit + 1) * T <= t_end;  // the segment holds the unit's last tile
         const bool with_kv = a.fused && closes;
@@ -368,7 +341,6 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         }
         // every cached row is read once per step: let it leave L2 first
         const uint64_t pol_stream = l2_policy_evict_first();
-        LAR_STAMP(1);
         int stage = pw;
         uint32_t empty_parity = 1;
         for (int i0 = 0; i0 < n_local; i0 += 32) {
@@ -382,13 +354,12 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             for (int i = 0; i < cnt; ++i) {
                 if (!dep_waited && kProducers * (i0 + i) + pw >= fill_end) {
                     grid_dep_wait();  // every tile from here on may still be written by the preceding kernels
-                    if (lane == 0) LAR_STAMP(2);
                     dep_waited = true;
                 }
                 const int yi = __shfl_sync(0xffffffffu, y, i), rti = __shfl_sync(0xffffffffu, rt, i);
                 if (lane == 0 && ok) {
                     const int ri = rti & 0xff;
-                    ok = LAR_WAIT(16, true, wait_or_abort(bar_empty + stage * 8, empty_parity, abort_flag));
+                    ok = wait_or_abort(bar_empty + stage * 8, empty_parity, abort_flag);
                     if (ok) {
                         const uint32_t bar = bar_full + stage * 8, dst = ring + (uint32_t)stage * TR::STAGE_BYTES;
                         if (ri > 0) {
@@ -409,7 +380,6 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             }
         }
         if (!dep_waited) grid_dep_wait();
-        LAR_STAMP(3);
         if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
     } else if (warp < kProducers + W) {
         // =========================================================================== consumers
@@ -428,9 +398,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
 
             // ---- Q fragments (A operand): row qrow = head, 16 columns per k-step; heads >= G are zero rows
             const int qs = seg % NQ;
-            const long long tq0 = LAR_CLK();
-            ok = LAR_WAIT(18, cw == 0, wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag));
-            if (cw == 0 && seg == 0) LAR_STAMP(4);
+            ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             uint32_t qa0[TR::KSTEPS], qa2[TR::KSTEPS];
             {
@@ -448,7 +416,6 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_qempty + qs * 8);
 
-            LAR_ACC(27, cw == 0, LAR_CLK() - tq0);
             // running maximum and this thread's share of the row sum of heads 2 quad and 2 quad + 1
             float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
             // O^T: o[t][0], o[t][1] = heads 2 quad, 2 quad + 1 at d = 16 t + qrow; o[t][2], o[t][3] at d + 8
@@ -458,8 +425,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
 
             for (; j < je; j += W) {
                 const int s = stage;
-                ok = LAR_WAIT(19, cw == 0, wait_or_abort(bar_full + s * 8, full_parity, abort_flag));
-                if (j == 0) LAR_STAMP(5);
+                ok = wait_or_abort(bar_full + s * 8, full_parity, abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
                 stage += W;
                 if (stage >= NS) {
@@ -469,7 +435,6 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                 const int tile = t_begin + j - ub;
                 const int rows = len - tile * kStreamTile < kStreamTile ? len - tile * kStreamTile : kStreamTile;
                 const uint32_t St = ring + (uint32_t)s * TR::STAGE_BYTES;
-                const long long tc0 = LAR_CLK();
                 if (rows > 0) {
                     const int box_rows = (rows + 3) & ~3;  // K rows are lines 0.., V rows lines box_rows.. of a block
                     // S^T[key][head] = K q^T for the 32 keys of the tile: the keys are the M rows (two 16-key tiles), the
@@ -545,16 +510,13 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_empty + s * 8);
-                LAR_ACC(23, cw == 0, LAR_CLK() - tc0);
-                LAR_ACC(24, cw == 0, 1);
             }
             if (!ok) break;
-            const long long ts0 = LAR_CLK();
 
             // ---- this warp's partial of the segment -> shared memory
             const int buf = seg % NPB;
             if (seg >= NPB) {
-                ok = LAR_WAIT(20, cw == 0, wait_or_abort(bar_pempty + buf * 8, (uint32_t)((seg / NPB - 1) & 1), abort_flag));
+                ok = wait_or_abort(bar_pempty + buf * 8, (uint32_t)((seg / NPB - 1) & 1), abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             }
 #pragma unroll
@@ -589,10 +551,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_pfull + buf * 8);
-            LAR_ACC(25, cw == 0, LAR_CLK() - ts0);
-            LAR_ACC(26, cw == 0, 1);
         }
-        if (cw == 0) LAR_STAMP(6);
         if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
     } else {
         // =========================================================================== epilogue
@@ -626,7 +585,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             const bool opens = ub >= t_begin, closes = ub + T <= t_end;
             const int qs = seg % NQ, buf = seg % NPB;
             closing_loads(seg + 1, page_nxt, dev_len_nxt);
-            ok = LAR_WAIT(21, true, wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag));
+            ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             const unsigned char* Qs = qring_ptr + qs * QENT;
             const uint16_t* Q16 = reinterpret_cast<const uint16_t*>(Qs);
@@ -698,9 +657,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             if (lane == 0) mbar_arrive(bar_qempty + qs * 8);
 
             // ---- merge the consumers' partials (+ the step's token)
-            ok = LAR_WAIT(22, true, wait_or_abort(bar_pfull + buf * 8, (uint32_t)((seg / NPB) & 1), abort_flag));
-            if (seg == 0) LAR_STAMP(7);
-            LAR_STAMP(9);
+            ok = wait_or_abort(bar_pfull + buf * 8, (uint32_t)((seg / NPB) & 1), abort_flag);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             const float* pb = pbuf + buf * pbuf_floats;
             // branch-free and unrolled over the (at most kMaxConsumers) consumer warps, so that the shared-memory
@@ -734,7 +691,6 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_pempty + buf * 8);
-            LAR_STAMP(10);
             // this segment's slot of the input ring is free once every consumer has taken its fragments: refill it
             if (lane == 0 && seg + NQ < n_segs) ok = issue_inputs(seg + NQ);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
@@ -765,7 +721,6 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                 int ticket = 0;
                 if (lane == 0) ticket = atomicAdd(a.tickets + unit, 1);
                 ticket = __shfl_sync(0xffffffffu, ticket, 0);
-                LAR_STAMP(11);
                 if (ticket == n_parts - 1) {
                     __threadfence();
                     // Heads in groups of GC, parts in pairs: the loads of a pair (m, l and the o row of every head
@@ -817,11 +772,9 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                         }
                     }
                     if (lane == 0) a.tickets[unit] = 0;
-                    LAR_STAMP(12);
                 }
             }
         }
-        LAR_STAMP(8);
         if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
     }
 

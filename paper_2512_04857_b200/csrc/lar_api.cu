@@ -913,18 +913,6 @@ lar_status_t lar_cache_get_state(lar_cache_t* c, int layer, int32_t* lens, int32
     return LAR_OK;
 }
 
-#ifdef LAR_TRACE
-// Trace builds only: copy the in-kernel timeline of the decode kernel (32 words per CTA) to the host and clear it.
-lar_status_t lar_debug_trace_read(unsigned long long* host_out, int n_ctas) {
-    if (!host_out || n_ctas != 1024) return LAR_ERR_INVALID_ARG;
-    LAR_CUDA(cudaDeviceSynchronize());
-    LAR_CUDA(cudaMemcpyFromSymbol(host_out, lar::lar_trace_buf, sizeof(unsigned long long) * 32 * 16 * (size_t)n_ctas));
-    static unsigned long long zeros[16 * 1024 * 32];
-    LAR_CUDA(cudaMemcpyToSymbol(lar::lar_trace_buf, zeros, sizeof(zeros)));
-    return LAR_OK;
-}
-#endif
-
 lar_status_t lar_cache_poll_device_status(lar_cache_t* c, uint32_t* bits_out, void* stream) {
     if (!c) return LAR_ERR_INVALID_ARG;
     LAR_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
