@@ -48,6 +48,23 @@ def whole_job_value(images_per_rank, n_visual, world, ms_per_step_max):
     return world * images_per_rank * n_visual / (ms_per_step_max * 1e-3)
 
 
+def _replica_entry(index, n, port, target, args):
+    os.environ.update({"RANK": str(index), "LOCAL_RANK": str(index), "WORLD_SIZE": str(n),
+                       "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
+    target(args)
+
+
+def spawn_replicas(n, target, args):
+    """`--gpus N` without a launcher: start N processes on this node, one replica per GPU, each with the
+    environment torchrun would give it (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR, MASTER_PORT)."""
+    import socket
+    import torch.multiprocessing as mp
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    mp.spawn(_replica_entry, args=(n, port, target, args), nprocs=n, join=True)
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -326,12 +343,14 @@ def time_generations(r: Runner, steps: int, warmup: int, dist=None, sampler=None
     return total_ms, decode_ms, clocks, (first_ms, last_ms)
 
 
-def measure_e2e(w, dev, args, steps=1):
+def measure_e2e(w, dev, args, steps=3):
     """Same metric through the host-buffer entry point: every layer-step copies q, k, v from pinned host
     memory, runs the fused kernel and copies the output back (all inside the timed region)."""
     import torch
     from paper_2512_04857_b200 import lar, workloads as W
     flags = lar.LAR_FLAG_NO_HOST_CHECKS | lar.LAR_FLAG_HOST_DEFER_OUT
+    if not args.no_pdl:
+        flags |= lar.LAR_FLAG_PDL
     cfg = lar.config_from_workload(w, flags=flags, kv_splits=args.kv_splits, warps_per_cta=args.warps,
                                    stages=args.stages, page_tokens=args.page_tokens, decode_ctas=args.ctas)
     cache = lar.Cache(cfg, device=str(dev))
@@ -358,10 +377,13 @@ def measure_e2e(w, dev, args, steps=1):
                 for t in range(n):
                     for layer in range(L):
                         cache.decode_step_host(layer, hq[t, layer], None, None, ho[t, layer])   # q | k | v packed
-                if kind == "line+end":
-                    for layer in range(L):
-                        cache.line_end_score_evict(layer)     # (per layer here: the host copies of a layer precede its kernels)
                 cache.host_join()                             # the line's last copy-outs re-join the stream
+                if kind == "line+end":
+                    if args.per_layer_line_end:
+                        for layer in range(L):
+                            cache.line_end_score_evict(layer)
+                    else:
+                        cache.line_end_score_evict_all()      # one launch for every layer, as in the headline
             graphs.append(g)
 
         def gen():
@@ -371,7 +393,8 @@ def measure_e2e(w, dev, args, steps=1):
                     cache.append_kv(layer, kc[layer], kc[layer], w.cond_len)
             for line in range(h):
                 graphs[0 if line < h - 1 else 1].replay()
-        gen()
+        for _ in range(2):
+            gen()
         torch.cuda.synchronize(dev)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
@@ -384,7 +407,7 @@ def measure_e2e(w, dev, args, steps=1):
     cache.close()
     qb = S * Hq * d * w.elt_bytes
     kb = S * Hkv * d * w.elt_bytes
-    return {"ms": ms, "h2d": w.n_visual * L * (qb + 2 * kb), "d2h": w.n_visual * L * qb, "status_bits": bits}
+    return {"ms": ms, "steps": steps, "h2d": w.n_visual * L * (qb + 2 * kb), "d2h": w.n_visual * L * qb, "status_bits": bits}
 
 
 def run_ours(args):
@@ -430,12 +453,21 @@ def run_ours(args):
         torch.cuda.empty_cache()
         return res
 
+    def roofline_of(wl, decode_ms_per_step):
+        kvb = wl.kv_bytes_per_generation()
+        nd = wl.n_visual * wl.n_layers
+        ach = kvb / (decode_ms_per_step * 1e-3) / 1e9
+        return {"bound": "hbm", "kernel": "decode_stream_kernel (fused append + decode attention)",
+                "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                "peak_kind": f"of {peak_kind} copy bandwidth", "frac_of_8TBs": ach / 8000.0,
+                "algorithmic_bytes_per_launch": kvb / nd, "avg_launch_us": decode_ms_per_step * 1e3 / nd,
+                "traffic": NCU_TRAFFIC_PER_LAUNCH.get(wl.name)}
+
     main = bench_workload(w, args.steps, args.warmup, True)
     ms_step, ms_decode = max_over_ranks([main["ms_per_step"], main["decode_ms_per_step"]], dist, dev)
     value = whole_job_value(w.images, w.n_visual, world, ms_step)
     kv_bytes = w.kv_bytes_per_generation()
     n_decode = w.n_visual * w.n_layers
-    achieved = kv_bytes / (ms_decode * 1e-3) / 1e9
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -452,19 +484,12 @@ def run_ours(args):
                        "plan": main["plan"], "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
             "clocks": main["clocks"],
             "gpu_launches": main["launches"] * args.steps,
-            "roofline": {"bound": "hbm", "kernel": "decode_stream_kernel (fused append + decode attention)",
-                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_kind": f"of {peak_kind} copy bandwidth",
-                         "frac_of_8TBs": achieved / 8000.0,
-                         "algorithmic_bytes_per_launch": kv_bytes / n_decode,
-                         "avg_launch_us": ms_decode * 1e3 / n_decode, "traffic": NCU_TRAFFIC_PER_LAUNCH.get(w.name)},
+            "roofline": roofline_of(w, ms_decode),
             "sequence_tokens_per_s": world * w.batch * w.n_visual / (ms_step * 1e-3),
             "line_end_ms_per_step": ms_step - ms_decode,
             "per_token_ms": {"first_half": main["per_token_ms_first_half"], "last_half": main["per_token_ms_last_half"]},
             "device_status_bits": main["status_bits"]}
 
-    if rank == 0 or dist is None:
-        pass
     # ---- speedup over the library's own full-cache path on the same inputs
     if not args.no_full:
         full = bench_workload(w.full_cache(), max(1, min(args.steps, 2)), 1, False)
@@ -483,19 +508,25 @@ def run_ours(args):
             dist.all_reduce(em, op=dist.ReduceOp.MAX)
         line["e2e"] = {"value": world * w.images * w.n_visual / (float(em[0]) * 1e-3), "unit": UNIT,
                        "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"], "ms_per_step": float(em[0]),
+                       "steps": e["steps"], "warmup": 2, "device_status_bits": e["status_bits"],
                        "api": "lar_decode_step_host (pinned host q|k|v -> device, kernel, out -> host) per layer-step; "
                               "copies on the library's own streams overlap the neighbouring calls' kernels (deferred copy-out, "
-                              "joined once per line), one CUDA graph per line"}
+                              "joined once per line), one CUDA graph per line, same launch configuration as the headline "
+                              "(programmatic dependent launch, one line-end launch for all layers)"}
     # ---- other benchmark shapes (not the headline line)
     if args.also:
         line["also"] = {}
         for name in args.also.split(","):
             w2 = W.WORKLOADS[name]
-            r2 = bench_workload(w2, max(1, min(args.steps, 3)), 1, False)
-            ach = w2.kv_bytes_per_generation() / (r2["decode_ms_per_step"] * 1e-3) / 1e9
-            line["also"][name] = {"value": world * w2.images * w2.n_visual / (r2["ms_per_step"] * 1e-3), "unit": UNIT,
-                                  "ms_per_step": r2["ms_per_step"], "roofline_achieved_gbs": ach,
-                                  "roofline_frac": ach / peak, "frac_of_8TBs": ach / 8000.0, "plan": r2["plan"]}
+            if name == w.name:
+                continue
+            n2 = max(1, min(args.steps, 3))
+            r2 = bench_workload(w2, n2, 3, True)
+            ms2, dec2 = max_over_ranks([r2["ms_per_step"], r2["decode_ms_per_step"]], dist, dev)
+            line["also"][name] = {"value": whole_job_value(w2.images, w2.n_visual, world, ms2), "unit": UNIT,
+                                  "ms_per_step": ms2, "steps": n2, "warmup": 3, "roofline": roofline_of(w2, dec2),
+                                  "line_end_ms_per_step": ms2 - dec2, "plan": r2["plan"], "clocks": r2["clocks"],
+                                  "device_status_bits": r2["status_bits"]}
     # ---- batch sweep of one shape, compressed and full-cache (not the headline line)
     if args.batch_sweep:
         wb = W.WORKLOADS[args.sweep_workload]
@@ -551,7 +582,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="janus_pro_7b")
-    ap.add_argument("--also", default="", help="comma-separated extra workloads reported under 'also'")
+    ap.add_argument("--also", default="gqa_1024",
+                    help="comma-separated extra workloads reported under 'also' with the headline's roofline fields "
+                         "(default: the 1024-px GQA shape, the other shape the target is stated on; '' for none)")
     ap.add_argument("--batch-sweep", default="", help="comma-separated image counts: sweep the batch of --sweep-workload")
     ap.add_argument("--sweep-workload", default="gqa_1024")
     ap.add_argument("--ratio-sweep", default="", help="comma-separated line budgets: sweep the budget of --sweep-workload")
@@ -574,6 +607,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_replicas(args.gpus, run_ours, args)   # plain `python bench.py --gpus N`: start the N replicas here
     else:
         run_ours(args)
 

@@ -211,7 +211,8 @@ lar_status_t lar_cache_get_state(lar_cache_t* c, int layer, int32_t* lens, int32
 /* Synchronises `stream` and returns LAR_ERR_DEVICE_CHECK if any kernel recorded a failed check since
  * the last poll (bits in *bits_out, may be NULL: 1 capacity, 2 line-end off boundary, 4 wait limit,
  * 8 decode on an empty cache, 16 the length the host passed to a decode kernel differs from
- * the device's, e.g. a captured graph replayed out of order); clears the word. */
+ * the device's, e.g. a captured graph replayed out of order, 32 a line end met a score that is not finite -- a NaN
+ * or Inf in a key or query; such entries rank lowest, exactly n are still evicted); clears the word. */
 lar_status_t lar_cache_poll_device_status(lar_cache_t* c, uint32_t* bits_out, void* stream);
 
 /* Enable (1) / disable (0) the host-side call-order checks at run time (see LAR_FLAG_NO_HOST_CHECKS). */
@@ -235,9 +236,9 @@ lar_status_t lar_cache_get_plan(const lar_cache_t* c, lar_plan_t* plan_out);
  *   q, out : device, bf16, [n_units, group, head_dim]      k, v : device, bf16, [n_units, len, head_dim], dense
  *   group 1..8, head_dim 64 or 128, len >= 1, softmax_scale 0 selects 1/sqrt(head_dim).
  *
- * Limits: n_units <= 16384 (one ticket per unit), otherwise LAR_ERR_CAPACITY and nothing is launched; the number of
- * key ranges per unit (at most 8) is reduced until n_units * ranges * group * (head_dim + 2) * 4 bytes fit into the
- * array, so larger problems run with fewer CTAs rather than fail.
+ * Limits: n_units <= 16384 (one ticket per unit), otherwise LAR_ERR_CAPACITY and nothing is launched.  A unit's keys
+ * are cut into at most 8 ranges (one CTA each) while n_units * ranges <= 296; the partials of such a launch take at
+ * most 1.3 MB of the array.  With more than 148 units every unit is one range and only the tickets are touched.
  * The call enqueues one memset (the tickets of the units it uses must start at zero; the array keeps whatever the
  * previous call left) and one kernel on `stream`, and calls no allocating routine.  The first call on a device looks
  * the array's device address up (cudaGetSymbolAddress, with that device current): make that first call outside any

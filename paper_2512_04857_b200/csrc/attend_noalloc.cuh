@@ -154,14 +154,17 @@ inline cudaError_t static_scratch_address(unsigned char** out) {
     return cudaSuccess;
 }
 
-// Key ranges per unit: enough CTAs for two per SM, at least 16 rows each, and the partials must fit.
-inline int static_scratch_splits(int n_units, int group, int head_dim, int len) {
-    int splits = 296 / n_units;
+// Key ranges per unit: enough CTAs for two per SM of a B200 and at least 16 rows each; with more than 148 units every
+// unit is one range and no partial is written.  n_units * ranges never exceeds kStaticMaxCtas, so the partials take at
+// most kStaticMaxCtas * 8 heads * (128 + 2) floats: they always fit behind the tickets.
+constexpr int kStaticMaxCtas = 296;
+static_assert((size_t)kStaticMaxCtas * 8 * (128 + 2) * sizeof(float) <= kStaticScratchBytes - kStaticTicketBytes,
+              "the partials of the largest split launch must fit into the static array");
+inline int static_scratch_splits(int n_units, int len) {
+    int splits = kStaticMaxCtas / n_units;
     if (splits > kStaticMaxSplits) splits = kStaticMaxSplits;
     if (splits > len / 16) splits = len / 16;
     if (splits < 1) splits = 1;
-    while (splits > 1 && (size_t)n_units * splits * group * (head_dim + 2) * sizeof(float) > kStaticScratchBytes - kStaticTicketBytes)
-        --splits;
     return splits;
 }
 

@@ -10,7 +10,7 @@ namespace lar {
 constexpr int kGranule = 16;  // rows of K (and V) moved by one bulk copy and processed as one tile
 
 // device status bits (lar_cache_poll_device_status)
-constexpr unsigned kStCapacity = 1u, kStBoundary = 2u, kStWaitLimit = 4u, kStEmpty = 8u, kStLength = 16u;
+constexpr unsigned kStCapacity = 1u, kStBoundary = 2u, kStWaitLimit = 4u, kStEmpty = 8u, kStLength = 16u, kStNonFinite = 32u;
 
 struct UnitState {
     int len;    // live entries (prefix + visual)

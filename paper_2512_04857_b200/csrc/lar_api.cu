@@ -675,6 +675,13 @@ lar_status_t lar_cache_reset(lar_cache_t* c, void* stream) {
     c->last_layer = -1;
     c->seq = 0;
     c->last_writer.assign(c->last_writer.size(), 0);
+    // host-buffer entry point: whatever was in flight is ordered before the reset on `stream` by the caller; forget it
+    for (int i = 0; i < kHostSlots; ++i) {
+        c->out_pending[i] = false;
+        c->slot_used[i] = false;
+        c->slot_capture[i] = 0;
+    }
+    c->last_host_capture = 0;
     return LAR_OK;
 }
 
@@ -748,6 +755,10 @@ lar_status_t lar_decode_step(lar_cache_t* c, int layer, const void* q, const voi
 lar_status_t lar_decode_step_host(lar_cache_t* c, int layer, const void* q_host, const void* k_host, const void* v_host,
                                   void* out_host, void* stream) {
     if (bad_layer(c, layer) || !q_host || !out_host || (!k_host) != (!v_host)) return LAR_ERR_INVALID_ARG;
+    {
+        const lar_status_t pre = check_visual_append(c, c->sh[layer]);  // before anything is enqueued
+        if (pre != LAR_OK) return pre;
+    }
     cudaStream_t s = (cudaStream_t)stream;
     const size_t qb = (size_t)c->cfg.batch * c->cfg.n_q_heads * c->d.row_bytes;
     const size_t kb = (size_t)c->cfg.batch * c->cfg.n_kv_heads * c->d.row_bytes;
@@ -855,7 +866,7 @@ lar_status_t lar_line_end_score_evict(lar_cache_t* c, int layer, void* stream) {
             lv, layer_strides(c), c->scale * 1.4426950408889634f, (c->cfg.flags & LAR_FLAG_SCORE_CACHE_NORM) ? 1 : 0);
         LAR_CUDA(cudaGetLastError());
         c->launches++;
-        c->last_layer = layer;
+        c->last_layer = -2;  // rows of the cache were just moved: the next decode launch must not fetch ahead
         c->last_writer[layer] = ++c->seq;
         if (sh.v >= c->d.B) sh.v -= c->cfg.line_width;
     }
@@ -931,7 +942,7 @@ lar_status_t lar_attend_dense_noalloc(const void* q, const void* k, const void* 
     if (n_units > lar::kStaticMaxUnits) return LAR_ERR_CAPACITY;  // one ticket per unit in the static array
     unsigned char* scratch = nullptr;
     LAR_CUDA(lar::static_scratch_address(&scratch));
-    const int splits = lar::static_scratch_splits(n_units, group, head_dim, len);
+    const int splits = lar::static_scratch_splits(n_units, len);
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
     cudaStream_t s = (cudaStream_t)stream;
     // the array keeps what the last call left: the tickets of this call must start at zero

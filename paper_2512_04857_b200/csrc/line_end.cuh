@@ -304,7 +304,16 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
         __syncthreads();
     }
 
-    // ---- Eq. 10: keep the M - n most salient; equal scores keep the lower slot (older token)
+    // ---- Eq. 10: keep the M - n most salient; equal scores keep the lower slot (older token).
+    // A score that is not finite (a NaN or Inf in a key or query) has no rank: it is treated as the lowest possible
+    // score, which keeps the ranking a total order and the kept count at M - n, and the status word records it.
+    for (int mm = tid; mm < M; mm += blockDim.x) {
+        if (!isfinite(S[mm])) {
+            S[mm] = -INFINITY;
+            atomicOr(lv.status, kStNonFinite);
+        }
+    }
+    __syncthreads();
     for (int mm = tid; mm < M; mm += blockDim.x) {
         const float s = S[mm];
         int rank = 0;
@@ -323,7 +332,7 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
             const int mm = m0 + lane;
             const bool kp = mm < M && keep[mm];
             const unsigned bal = __ballot_sync(0xffffffffu, kp);
-            if (kp) srcmap[base + __popc(bal & ((1u << lane) - 1u))] = mm;
+            if (kp && base + __popc(bal & ((1u << lane) - 1u)) < n_keep) srcmap[base + __popc(bal & ((1u << lane) - 1u))] = mm;
             base += __popc(bal);
         }
     }

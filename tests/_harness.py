@@ -9,6 +9,7 @@ oracle is then re-synchronised by evicting the GPU's choice so later steps compa
 """
 from __future__ import annotations
 
+import os
 from dataclasses import dataclass, field
 from typing import Dict, List, Optional, Sequence, Tuple
 
@@ -21,6 +22,21 @@ from paper_2512_04857_b200 import workloads as W
 
 TOL = {"bf16": 2e-2, "fp32": 1e-4}       # max-abs tolerance of attention outputs
 NEAR_TIE_REL = 1e-5
+# per test file: what the parity runs of this session compared (printed at the end of a pytest run)
+TOTALS: Dict[str, Dict[str, float]] = {}
+
+
+def _account(rep: "ParityReport") -> None:
+    where = os.environ.get("PYTEST_CURRENT_TEST", "outside pytest").split("::")[0]
+    t = TOTALS.setdefault(where, {"runs": 0, "outputs": 0, "line_ends": 0, "compressions": 0, "near_ties": 0,
+                                  "max_abs_err_bf16": 0.0, "max_abs_err_fp32": 0.0})
+    t["runs"] += 1
+    t["outputs"] += rep.outputs_compared
+    t["line_ends"] += rep.line_ends_compared
+    t["compressions"] += rep.compressions
+    t["near_ties"] += rep.near_ties
+    key = "max_abs_err_" + rep.dtype
+    t[key] = max(t[key], rep.max_abs_err)
 
 
 @dataclass
@@ -32,6 +48,7 @@ class ParityReport:
     near_ties: int = 0
     max_score_rel_err: float = 0.0
     mismatches: List[str] = field(default_factory=list)
+    dtype: str = "bf16"
 
     def ok(self, tol: float) -> bool:
         return not self.mismatches and self.max_abs_err <= tol
@@ -52,7 +69,7 @@ def run_parity(w: W.Workload, *, units: Optional[Sequence[Tuple[int, int, int]]]
     dev = torch.device(device)
     cfg = lar.config_from_workload(w, **(cfg_overrides or {}))
     cache = lar.Cache(cfg, device=device)
-    rep = ParityReport()
+    rep = ParityReport(dtype=w.dtype)
     L, S, Hq, Hkv, d, G, n, C = (w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.group,
                                  w.line_width, w.cond_len)
     N = w.n_visual if n_steps is None else n_steps
@@ -171,4 +188,5 @@ def run_parity(w: W.Workload, *, units: Optional[Sequence[Tuple[int, int, int]]]
     for u in orc.values():
         u.close()
     cache.close()
+    _account(rep)
     return rep

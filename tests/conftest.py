@@ -36,3 +36,24 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter, exitstatus, config):
+    """What the parity runs compared with the oracle, and how many kept sets differed from it only at score near-ties
+    (oracle scores within 1e-5 relative of the eviction boundary): the count is reported, not just bounded."""
+    try:
+        from _harness import TOTALS
+    except Exception:
+        return
+    if not TOTALS:
+        return
+    tr = terminalreporter
+    tr.write_sep("-", "parity against the CPU oracle")
+    tot_c = tot_n = 0
+    for where, t in sorted(TOTALS.items()):
+        tot_c += t["compressions"]
+        tot_n += t["near_ties"]
+        tr.write_line(f"{where}: {t['runs']} runs, {t['outputs']} output elements, {t['line_ends']} line ends, "
+                      f"{t['compressions']} compressions compared, {t['near_ties']} near-ties, "
+                      f"max abs err bf16 {t['max_abs_err_bf16']:.3e} fp32 {t['max_abs_err_fp32']:.3e}")
+    tr.write_line(f"near-ties: {tot_n} of {tot_c} compressions compared")

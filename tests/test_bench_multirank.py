@@ -48,6 +48,34 @@ def test_two_ranks_take_the_slowest_time_and_the_whole_job_value():
         assert value == pytest.approx(2 * 16 * 576 / 15e-3)
 
 
+def _stub_replica(args):
+    """What a replica does around its measurement, without a GPU: join the job from the environment that
+    spawn_replicas prepared, agree on the slowest time, and let rank 0 write the line."""
+    sys.path.insert(0, ROOT)
+    import json
+    import bench
+    rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+    assert int(os.environ["LOCAL_RANK"]) == rank
+    dist.init_process_group(backend="gloo")
+    ms = bench.max_over_ranks([100.0 + 50.0 * rank], dist, torch.device("cpu"))[0]
+    dist.barrier()
+    if rank == 0:
+        with open(args["out"], "w") as f:
+            json.dump({"n_gpus": world, "ms_per_step": ms, "value": bench.whole_job_value(16, 576, world, ms)}, f)
+    dist.destroy_process_group()
+
+
+def test_gpus_flag_without_a_launcher_starts_the_replicas(tmp_path):
+    sys.path.insert(0, ROOT)
+    import json
+    import bench
+    out = tmp_path / "line.json"
+    bench.spawn_replicas(2, _stub_replica, {"out": str(out)})
+    line = json.loads(out.read_text())
+    assert line["n_gpus"] == 2 and line["ms_per_step"] == 150.0
+    assert line["value"] == pytest.approx(2 * 16 * 576 / 0.150)
+
+
 def test_single_process_is_the_identity():
     sys.path.insert(0, ROOT)
     import bench

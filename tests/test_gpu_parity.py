@@ -152,6 +152,41 @@ def test_full_size_shapes_sampled_units(name, layers, n_units):
     assert rep.compressions == n_units * (w.n_lines - w.budget_lines)
 
 
+def _with_budget(w, lines):
+    """The benchmark's budget sweep: N_init = n, r = (budget_lines - 2) / 2 (at least 1)."""
+    return w.scaled(budget_lines=lines, recent_lines=max(1, (lines - 2) // 2), anchor_len=w.line_width)
+
+
+# every configuration a benchmark number is quoted on: the efficiency table's batch sizes (256 / 64 / 12 images) and
+# budget ratios (1/4, 1/6, 1/8), the batch-sweep end points of the 1024-px shape, and the two added model shapes
+QUOTED = {
+    "janus_pro_7b at 64 images": lambda: W.WORKLOADS["janus_pro_7b"].scaled(batch=128, images=64),
+    "gqa_1024 at 64 images": lambda: W.WORKLOADS["gqa_1024"].scaled(batch=128, images=64),
+    "gqa_1024 at 1 image": lambda: W.WORKLOADS["gqa_1024"].scaled(batch=2, images=1),
+    "llamagen_xl at 256 images": lambda: W.WORKLOADS["llamagen_xl"].scaled(batch=512, images=256),
+    "lumina_768 at 12 images": lambda: W.WORKLOADS["lumina_768"].scaled(batch=24, images=12),
+    "llamagen_xxl": lambda: W.WORKLOADS["llamagen_xxl"],
+    "janus_pro_1b": lambda: W.WORKLOADS["janus_pro_1b"],
+    "janus_pro_7b budget 6 lines (1/4)": lambda: _with_budget(W.WORKLOADS["janus_pro_7b"], 6),
+    "janus_pro_7b budget 3 lines (1/8)": lambda: _with_budget(W.WORKLOADS["janus_pro_7b"], 3),
+    "llamagen_xl budget 6 lines (1/4)": lambda: _with_budget(W.WORKLOADS["llamagen_xl"], 6),
+    "lumina_768 budget 12 lines (1/4)": lambda: _with_budget(W.WORKLOADS["lumina_768"], 12),
+    "lumina_768 budget 8 lines (1/6)": lambda: _with_budget(W.WORKLOADS["lumina_768"], 8),
+}
+
+
+@pytest.mark.parametrize("which", sorted(QUOTED))
+def test_quoted_configurations_sampled_units(which):
+    """One layer (layers are independent and identically shaped; the launch plan does not depend on their number), the
+    whole generation in the benchmark's launch configuration, the oracle on a sample of units."""
+    w = QUOTED[which]().scaled(n_layers=1)
+    n_units = 3
+    rep = run_parity(w, units=pick_units(w, n_units, seed=5), gen_device="cuda",
+                     cfg_overrides=dict(flags=lar.LAR_FLAG_PDL), line_end_all=True)
+    _check(rep, w, allow_near_ties=2)
+    assert rep.compressions == min(n_units, w.batch * w.n_kv_heads) * (w.n_lines - w.budget_lines)
+
+
 @pytest.mark.parametrize("name,steps", [("janus_pro_7b", None), ("gqa_1024", 65 * 20)])
 def test_full_cache_path_full_size_sampled(name, steps):
     w = W.WORKLOADS[name].scaled(n_layers=1).full_cache()
@@ -219,7 +254,7 @@ def test_bf16_mid_region_smaller_than_one_key_tile():
 
 
 # ------------------------------------------------------------------ every layer of the deepest shapes
-@pytest.mark.parametrize("name", ["janus_pro_7b", "gqa_1024"])
+@pytest.mark.parametrize("name", ["janus_pro_7b", "gqa_1024", "llamagen_xl", "lumina_768"])
 def test_every_layer_of_the_full_size_shape(name):
     """All layers, full batch, whole generation in the benchmark's launch configuration (fused step, PDL, one
     line-end launch for all layers); the oracle follows one unit of every layer (sequence and head vary with the layer)."""

@@ -95,6 +95,51 @@ def test_device_side_checks_record_status_instead_of_faulting():
     c.close()
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_a_key_that_is_not_finite_is_recorded_and_the_line_end_still_evicts_n(dtype):
+    """A NaN key gives NaN scores: they rank lowest, the kept count stays M - n (the length trajectory is unchanged, the
+    index map has no duplicate) and status bit 32 tells the host."""
+    cfg = _small(n_layers=1, dtype=dtype, budget_lines=4, n_lines=8)     # B = 32, N_init = 8, r = 1: M = 16, evict 8
+    c = lar.Cache(cfg)
+    b = _bufs(cfg)
+    c.append_kv(0, b["kc"], b["vc"], 4)
+    g = torch.Generator(device="cpu").manual_seed(7)
+    for t in range(32):
+        k = torch.randn(cfg.batch, cfg.n_kv_heads, cfg.head_dim, generator=g).to(b["k"].dtype).to("cuda:0")
+        if t == 12:                                    # a mid token (visual index 13: behind the anchor, before the last line)
+            k[0, 1, 5] = float("nan")
+        c.decode_step(0, b["q"], k, b["v"], b["out"])
+        if t % 8 == 7:
+            c.line_end_score_evict(0)
+    bits = c.poll_device_status()
+    assert bits == 32, bits
+    lens, imap = c.get_state(0)
+    assert (lens == 4 + 32 - 8).all()
+    for u in range(cfg.batch * cfg.n_kv_heads):
+        live = imap[u, : lens[u]]
+        assert len(set(live.tolist())) == len(live) and (np.diff(live) > 0).all()
+    # (a NaN key poisons the softmax of every guide row of its unit: all its scores tie at the bottom, so the n
+    # newest mid tokens go, as for any tie)
+    assert imap[1, : lens[1]].tolist() == list(range(4 + 16)) + list(range(4 + 24, 4 + 32))
+    c.close()
+
+
+def test_reset_forgets_deferred_host_copies():
+    cfg = _small(n_layers=1, flags=lar.LAR_FLAG_HOST_DEFER_OUT)
+    c = lar.Cache(cfg)
+    b = _bufs(cfg)
+    hq = torch.cat([b["q"].flatten(), b["k"].flatten(), b["v"].flatten()]).cpu().pin_memory()
+    ho = torch.empty(b["out"].shape, dtype=b["out"].dtype).pin_memory()
+    for _ in range(2):                                 # second round: the slots' bookkeeping starts afresh
+        c.append_kv(0, b["kc"], b["vc"], 4)
+        for _ in range(3):
+            c.decode_step_host(0, hq, None, None, ho)
+        torch.cuda.synchronize()
+        c.reset()
+    assert c.poll_device_status() == 0
+    c.close()
+
+
 def test_host_buffer_entry_point_matches_device_entry_point():
     cfg = _small(n_layers=1)
     b = _bufs(cfg)

@@ -5,15 +5,33 @@ framework's "no allocation" region, a server whose KV-cache manager already owns
 receives raw pointers.  They have no slab to give, so this call keeps its split-KV partials in a static device array
 of the library.  The test drives the ordinary cache entry point (lar_decode_step) and the no-allocation call on the
 same keys and values, two steps in a row, and checks that both give the same attention output within the bf16
-tolerance of the parity tests.  It runs last (file name) so that a failure here cannot hide other results."""
+tolerance of the parity tests -- and that the no-allocation call agrees with the CPU oracle's Eq. 2 on the same bf16
+inputs within that tolerance.  It runs last (file name) so that a failure here cannot hide other results."""
+import numpy as np
 import pytest
 import torch
 
+from oracle import lar_oracle as O
 from paper_2512_04857_b200 import lar
 
 pytestmark = pytest.mark.gpu
 
 TOL_BF16 = 2e-2     # max-abs tolerance of bf16 attention outputs, as in the parity tests
+
+
+def _against_oracle(q, k_all, v_all, out, group, head_dim, sample=5):
+    """max-abs difference to the oracle's attention (fp64, Eq. 2) on a few units."""
+    units = k_all.shape[0] * k_all.shape[1]
+    qf = q.reshape(units, group, head_dim).float().cpu().numpy()
+    kf = k_all.reshape(units, -1, head_dim).float().cpu().numpy()
+    vf = v_all.reshape(units, -1, head_dim).float().cpu().numpy()
+    of = out.reshape(units, group, head_dim).float().cpu().numpy().astype(np.float64)
+    worst = 0.0
+    for u in sorted({0, units - 1, *range(0, units, max(1, units // sample))}):
+        for g in range(group):
+            ref = O.attention(qf[u, g], kf[u], vf[u], 1.0 / np.sqrt(head_dim))
+            worst = max(worst, float(np.max(np.abs(of[u, g] - ref))))
+    return worst
 
 
 def _run(head_dim, n_q_heads, n_kv_heads, cond_len, batch=3):
@@ -44,6 +62,7 @@ def _run(head_dim, n_q_heads, n_kv_heads, cond_len, batch=3):
         torch.cuda.synchronize()
         assert torch.isfinite(out.float()).all()
         worst = max(worst, (out.float() - ref.float()).abs().max().item())
+        worst = max(worst, _against_oracle(q, k_all, v_all, out, group, head_dim))
     assert cache.poll_device_status() == 0
     cache.close()
     return worst
@@ -52,10 +71,16 @@ def _run(head_dim, n_q_heads, n_kv_heads, cond_len, batch=3):
 @pytest.mark.parametrize("head_dim,n_q_heads,n_kv_heads,cond_len", [
     (128, 8, 8, 200),      # several key ranges per unit: partials and tickets in the static array
     (64, 8, 2, 37),        # grouped queries, ragged length
-    (128, 4, 4, 3),        # shorter than one key range: no scratch used
+    (128, 4, 4, 3),        # shorter than one key range (fewer than 16 rows): no scratch used
+    (128, 8, 1, 200),      # 8 query heads per KV head, 8 key ranges per unit: the largest partials
 ])
 def test_no_alloc_entry_point_matches_cache_entry_point(head_dim, n_q_heads, n_kv_heads, cond_len):
     assert _run(head_dim, n_q_heads, n_kv_heads, cond_len) <= TOL_BF16
+
+
+def test_no_alloc_entry_point_with_more_units_than_ctas_can_be_split():
+    """More than 296 units of 70 rows: every unit is one key range, only the tickets of the static array are touched."""
+    assert _run(64, 40, 20, 68, batch=16) <= TOL_BF16     # 320 units
 
 
 def test_no_alloc_entry_point_rejects_what_does_not_fit():
