@@ -371,14 +371,20 @@ def measure_e2e(w, dev, args, steps=3):
     s = torch.cuda.Stream(device=dev)
     graphs = []
     with torch.cuda.stream(s):
-        for kind in ("line+end", "line"):
+        # one graph per line, captured in order (a graph holds the cache lengths of the steps it was captured at)
+        for line in range(h):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=s):
+                if line == 0:
+                    cache.reset()
+                    if w.cond_len:
+                        for layer in range(L):
+                            cache.append_kv(layer, kc[layer], kc[layer], w.cond_len)
                 for t in range(n):
                     for layer in range(L):
                         cache.decode_step_host(layer, hq[t, layer], None, None, ho[t, layer])   # q | k | v packed
                 cache.host_join()                             # the line's last copy-outs re-join the stream
-                if kind == "line+end":
+                if line < h - 1 and not w.is_full_cache:
                     if args.per_layer_line_end:
                         for layer in range(L):
                             cache.line_end_score_evict(layer)
@@ -387,12 +393,8 @@ def measure_e2e(w, dev, args, steps=3):
             graphs.append(g)
 
         def gen():
-            cache.reset()
-            if w.cond_len:
-                for layer in range(L):
-                    cache.append_kv(layer, kc[layer], kc[layer], w.cond_len)
-            for line in range(h):
-                graphs[0 if line < h - 1 else 1].replay()
+            for g in graphs:
+                g.replay()
         for _ in range(2):
             gen()
         torch.cuda.synchronize(dev)

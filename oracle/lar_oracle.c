@@ -22,7 +22,10 @@
  *   - first compression happens at the end of line B/n (cache exactly full).
  *   - N_init and r are parameters (their values are not in the paper's main text).
  *   - the softmax of Eq. 9 normalises over the mid keys only, as the equation is written
- *     (score_norm = 1 selects the other reading: the probabilities the queries had at decode time).
+ *     (score_norm = 1 selects the other reading: the probabilities the queries had at decode time;
+ *     score_norm = 2 the accumulated-attention scoring of the paper's ablation "w. AttAcc" and of the
+ *     H2O-style baselines it describes: every cached token's attention probability of Eq. 2-3, summed
+ *     over all decode steps since the token was appended and over the G heads).
  *   - with grouped-query attention the score of a cached token is the mean over the G query heads
  *     that share its KV head (folded into the 1/n of Eq. 9 as 1/(nG)).
  *   - ties in BottomK: among equal scores the token with the higher original position is evicted
@@ -52,7 +55,11 @@ typedef struct {
     int head_dim;      /* d      */
     double scale;      /* logit scale; 0 selects 1/sqrt(d) */
     int score_norm;    /* 0: Eq. 9 as written (softmax over the mid keys only);
-                          1: variant -- softmax over every entry the query attended to when it was decoded */
+                          1: variant -- softmax over every entry the query attended to when it was decoded;
+                          2: accumulated attention over all history (the "w. AttAcc" ablation): the score of an
+                             entry is the sum of the probabilities Eq. 2-3 gave it at every step since it was
+                             appended, over the G heads, divided by n G (so that a sum that restarted at every
+                             line end would equal variant 1) */
 } lar_oracle_cfg;
 
 typedef struct {
@@ -64,6 +71,7 @@ typedef struct {
     int *pos;         /* [cap] original position: prefix j -> j, visual token i (1-based) -> C + i - 1 */
     double *K, *V;    /* [cap][d] */
     double *guide;    /* [n][G][d] */
+    double *acc;      /* [cap] attention mass each live entry has received so far (score_norm = 2) */
 } lar_oracle_unit;
 
 static double cfg_scale(const lar_oracle_cfg *c) {
@@ -189,18 +197,24 @@ lar_oracle_unit *lar_oracle_unit_create(const lar_oracle_cfg *cfg) {
     u->K = (double *)calloc((size_t)u->cap * d, sizeof(double));
     u->V = (double *)calloc((size_t)u->cap * d, sizeof(double));
     u->guide = (double *)calloc((size_t)cfg->line_width * (size_t)cfg->group * d, sizeof(double));
+    u->acc = (double *)calloc((size_t)u->cap, sizeof(double));
     return u;
 }
 
 void lar_oracle_unit_destroy(lar_oracle_unit *u) {
     if (!u) return;
-    free(u->pos); free(u->K); free(u->V); free(u->guide); free(u);
+    free(u->pos); free(u->K); free(u->V); free(u->guide); free(u->acc); free(u);
 }
 
 int lar_oracle_unit_len(const lar_oracle_unit *u) { return u->len; }
 int lar_oracle_unit_n_visual(const lar_oracle_unit *u) { return u->n_vis; }
 void lar_oracle_unit_positions(const lar_oracle_unit *u, int *pos_out) {
     memcpy(pos_out, u->pos, sizeof(int) * (size_t)u->len);
+}
+
+/* Attention mass every live entry has received since it was appended (cache order), summed over the G heads. */
+void lar_oracle_unit_accumulated(const lar_oracle_unit *u, double *acc_out) {
+    memcpy(acc_out, u->acc, sizeof(double) * (size_t)u->len);
 }
 
 /* Prefill (Sec. 3.1): the C conditional K/V rows become entries 0..C-1.  kc, vc: [C][d] floats. */
@@ -235,13 +249,17 @@ int lar_oracle_unit_step(lar_oracle_unit *u, const float *q, const float *k, con
     for (int t = 0; t < d; ++t) { u->K[(size_t)s * d + t] = (double)k[t]; u->V[(size_t)s * d + t] = (double)v[t]; }
     u->len += 1;
     u->n_vis += 1;
+    u->acc[s] = 0.0;                       /* a new entry has received no attention yet */
     double *qd = (double *)malloc(sizeof(double) * (size_t)d);
+    double *pr = (double *)malloc(sizeof(double) * (size_t)u->len);
     for (int g = 0; g < G; ++g) {
         for (int t = 0; t < d; ++t) qd[t] = (double)q[(size_t)g * d + t];
-        lar_oracle_attention(qd, u->K, u->V, u->len, d, cfg_scale(c), out + (size_t)g * d,
-                             probs ? probs + (size_t)g * u->len : NULL);
+        lar_oracle_attention(qd, u->K, u->V, u->len, d, cfg_scale(c), out + (size_t)g * d, pr);
+        if (probs) memcpy(probs + (size_t)g * u->len, pr, sizeof(double) * (size_t)u->len);
+        for (int j = 0; j < u->len; ++j) u->acc[j] += pr[j];   /* accumulated attention of every live entry */
         memcpy(u->guide + ((size_t)u->n_guide * G + g) * d, qd, sizeof(double) * (size_t)d);
     }
+    free(pr);
     free(qd);
     u->n_guide += 1;
     return 0;
@@ -289,6 +307,8 @@ int lar_oracle_unit_mid_scores(const lar_oracle_unit *u, double *scores, int *mi
     /* all n * G guide rows contribute equally: mean over the n queries and the G heads */
     if (c->score_norm == 0)
         lar_oracle_saliency(u->guide, c->line_width * c->group, Kmid, M, d, cfg_scale(c), scores);
+    else if (c->score_norm == 2)   /* the attention mass the entry has received since it was appended */
+        for (int m = 0; m < M; ++m) scores[m] = u->acc[slots[m]] / (double)(c->line_width * c->group);
     else   /* query t of the line is visual token n_vis - n + t + 1, at position C + n_vis - n + t */
         lar_oracle_saliency_cache(u->guide, c->line_width, c->group, u->K, u->pos, u->len, d, cfg_scale(c),
                                   c->cond_len + u->n_vis - c->line_width, slots, M, scores);
@@ -317,6 +337,7 @@ int lar_oracle_unit_evict(lar_oracle_unit *u, const int *evict_pos, int n_evict)
             if (drop[s]) continue;
             if (w != s) {
                 u->pos[w] = u->pos[s];
+                u->acc[w] = u->acc[s];   /* an entry keeps the attention it has accumulated */
                 memcpy(u->K + (size_t)w * d, u->K + (size_t)s * d, sizeof(double) * (size_t)d);
                 memcpy(u->V + (size_t)w * d, u->V + (size_t)s * d, sizeof(double) * (size_t)d);
             }

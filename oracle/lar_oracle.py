@@ -46,6 +46,8 @@ def lib():
             getattr(L, name).restype = C.c_int
         L.lar_oracle_unit_positions.argtypes = [C.c_void_p, ip]
         L.lar_oracle_unit_positions.restype = None
+        L.lar_oracle_unit_accumulated.argtypes = [C.c_void_p, dp]
+        L.lar_oracle_unit_accumulated.restype = None
         L.lar_oracle_unit_prefill.argtypes = [C.c_void_p, fp, fp]
         L.lar_oracle_unit_prefill.restype = C.c_int
         L.lar_oracle_unit_step.argtypes = [C.c_void_p, fp, fp, fp, dp, dp]
@@ -83,6 +85,10 @@ def _f64(x):
     return np.ascontiguousarray(np.asarray(x, dtype=np.float64))
 
 
+# Eq. 9 as written / softmax over the whole live cache / attention accumulated over all history
+SCORE_NORM = {"mid": 0, "cache": 1, "accum": 2}
+
+
 def make_cfg(cond_len, line_width, n_lines, budget_lines, anchor_len, recent_lines, group, head_dim,
              scale=0.0, score_norm=0) -> Cfg:
     return Cfg(cond_len, line_width, n_lines, budget_lines, anchor_len, recent_lines, group, head_dim,
@@ -91,7 +97,7 @@ def make_cfg(cond_len, line_width, n_lines, budget_lines, anchor_len, recent_lin
 
 def cfg_from_workload(w) -> Cfg:
     return make_cfg(w.cond_len, w.line_width, w.n_lines, w.budget_lines, w.anchor_len, w.recent_lines,
-                    w.group, w.head_dim, score_norm=1 if getattr(w, "score_norm", "mid") == "cache" else 0)
+                    w.group, w.head_dim, score_norm=SCORE_NORM[getattr(w, "score_norm", "mid")])
 
 
 def attention(q, K, V, scale, want_probs=False):
@@ -165,6 +171,12 @@ class Unit:
         p = np.zeros(max(self.len, 1), dtype=np.int32)
         lib().lar_oracle_unit_positions(self._h, _i(p))
         return p[: self.len]
+
+    def accumulated(self) -> np.ndarray:
+        """Attention mass each live entry has received since it was appended (cache order; sum over the G heads)."""
+        a = np.zeros(max(self.len, 1))
+        lib().lar_oracle_unit_accumulated(self._h, _d(a))
+        return a[: self.len]
 
     def prefill(self, kc, vc):
         kc, vc = _f32(kc), _f32(vc)

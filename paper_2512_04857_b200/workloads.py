@@ -55,7 +55,8 @@ class Workload:
     seed: int
     prefix_key_scale: float = 1.0
     note: str = ""
-    score_norm: str = "mid"  # softmax of Eq. 9 over the "mid" keys (as written) or over the whole live "cache" (variant)
+    score_norm: str = "mid"  # scoring at a line end: Eq. 9 over the "mid" keys (as written), over the whole live "cache"
+                             # (variant), or "accum": attention accumulated over all decode steps (the paper's ablation)
 
     @property
     def n_visual(self) -> int:            # N

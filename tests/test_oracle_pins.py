@@ -402,3 +402,130 @@ def test_the_two_normalisations_differ_and_can_change_the_kept_set():
     assert (p0 == p1).all()
     assert abs(S0.sum() - 1.0) < 1e-9 and S1.sum() < 0.9
     assert not np.allclose(S0 / S0.sum(), S1 / S1.sum(), rtol=1e-3)
+
+
+# ------------------------------------------------- accumulated attention over all history (the "w. AttAcc" ablation)
+def _drive_generation(cfg, seed, on_step=None, on_line_end=None):
+    """Prefill and decode a whole image; calls on_step(u, i, probs) after step i (0-based) and
+    on_line_end(u, line) before every line end that is followed by another line."""
+    r = np.random.default_rng(seed)
+    C_, n, h, G, d = cfg.cond_len, cfg.line_width, cfg.n_lines, cfg.group, cfg.head_dim
+    u = O.Unit(cfg)
+    u.prefill(r.normal(size=(C_, d)), r.normal(size=(C_, d)))
+    for i in range(n * h):
+        _, probs = u.step(r.normal(size=(G, d)), r.normal(size=d), r.normal(size=d), want_probs=True)
+        if on_step:
+            on_step(u, i, probs)
+        if (i + 1) % n == 0 and (i + 1) < n * h:
+            if on_line_end:
+                on_line_end(u, (i + 1) // n)
+            u.line_end()
+    return u
+
+
+@pytest.mark.parametrize("G", [1, 2])
+def test_accumulated_scores_are_the_decode_probabilities_summed_since_the_append(G):
+    # the probabilities every step returns (Eq. 2-3, pinned to the library softmax above) are accumulated here per
+    # original position; at every compressing line end the oracle's scores must be those sums / (n G), and an evicted
+    # entry must never come back
+    cfg = O.make_cfg(3, 4, 9, 4, 2, 1, G, 8, score_norm=2)
+    mass = {}
+    seen_compressions = [0]
+
+    def on_step(u, i, probs):
+        for s, p in enumerate(u.positions()):
+            mass[int(p)] = mass.get(int(p), 0.0) + float(probs[:, s].sum())
+
+    def on_line_end(u, line):
+        if u.line_end_due() == 1:
+            S, mid_pos = u.mid_scores()
+            expect = np.array([mass[int(p)] for p in mid_pos]) / (cfg.line_width * G)
+            np.testing.assert_allclose(S, expect, rtol=1e-12, atol=1e-15)
+            seen_compressions[0] += 1
+
+    _drive_generation(cfg, 11, on_step, on_line_end)
+    assert seen_compressions[0] == cfg.n_lines - cfg.budget_lines
+
+
+def test_accumulated_scores_are_the_sum_over_lines_of_the_cache_normalised_scores():
+    # another route to the same numbers: at the end of every line (compressing or not) the cache-normalised form of
+    # Eq. 9 (pinned to the library softmax with a causal cut above), taken over ALL live entries, gives each entry's
+    # mean probability over that line; summed over the lines an entry has lived through this is its accumulated score
+    cfg = O.make_cfg(2, 3, 8, 4, 3, 1, 2, 8, score_norm=2)
+    n, G = cfg.line_width, cfg.group
+    total = {}
+    checked = [0]
+    guide = []
+
+    def on_step(u, i, probs):
+        pass
+
+    r = np.random.default_rng(23)
+    C_, h, d = cfg.cond_len, cfg.n_lines, cfg.head_dim
+    u = O.Unit(cfg)
+    Ks = {}
+    kc = r.normal(size=(C_, d))
+    u.prefill(kc, r.normal(size=(C_, d)))
+    for j in range(C_):
+        Ks[j] = kc[j].astype(np.float32).astype(np.float64)
+    for i in range(n * h):
+        q, k = r.normal(size=(G, d)), r.normal(size=d)
+        u.step(q, k, r.normal(size=d))
+        Ks[C_ + i] = k.astype(np.float32).astype(np.float64)
+        guide.append(q.astype(np.float32).astype(np.float64))
+        if (i + 1) % n == 0 and (i + 1) < n * h:
+            pos = u.positions()
+            K = np.stack([Ks[int(p)] for p in pos])
+            S_line = O.saliency_cache(np.stack(guide[-n:]), K, pos, C_ + i + 1 - n, list(range(len(pos))),
+                                      1.0 / np.sqrt(d))
+            for s, p in enumerate(pos):
+                total[int(p)] = total.get(int(p), 0.0) + float(S_line[s])
+            if u.line_end_due() == 1:
+                S, mid_pos = u.mid_scores()
+                np.testing.assert_allclose(S, [total[int(p)] for p in mid_pos], rtol=1e-10, atol=1e-14)
+                checked[0] += 1
+            u.line_end()
+    assert checked[0] == h - cfg.budget_lines
+
+
+def test_accumulated_attention_mass_is_conserved():
+    # every step hands out exactly one unit of probability per head: the mass on the live entries plus the mass the
+    # evicted entries took with them is G times the number of steps
+    cfg = O.make_cfg(4, 5, 7, 3, 5, 1, 3, 8, score_norm=2)
+    gone = [0.0]
+    state = {}
+
+    def on_line_end(u, line):
+        state["before"] = dict(zip((int(p) for p in u.positions()), u.accumulated()))
+
+    def on_step(u, i, probs):
+        if "before" in state and (i % cfg.line_width) == 0 and i > 0:
+            live = set(int(p) for p in u.positions())
+            gone[0] += sum(a for p, a in state.pop("before").items() if p not in live)
+        assert abs(u.accumulated().sum() + gone[0] - cfg.group * (i + 1)) < 1e-9
+
+    u = _drive_generation(cfg, 31, on_step, on_line_end)
+    assert gone[0] > 0.0 and u.len == cfg.cond_len + cfg.budget_lines * cfg.line_width
+
+
+def test_accumulated_scoring_keeps_a_heavy_hitter_that_the_line_scores_would_drop():
+    # one early key attracts every query of the first lines and none of the last line before the first compression:
+    # its accumulated score is the largest of the mid region, its Eq. 9 score among the smallest
+    cfgs = {sn: O.make_cfg(0, 4, 8, 5, 4, 1, 1, 4, scale=1.0, score_norm=sn) for sn in (0, 2)}
+    kept = {}
+    for sn, cfg in cfgs.items():
+        u = O.Unit(cfg)
+        u.prefill(np.zeros((0, 4)), np.zeros((0, 4)))
+        n = cfg.line_width
+        for i in range(cfg.budget_lines * n):
+            k = np.zeros(4)
+            k[1] = 0.01 * i                                # distinct, weak keys
+            if i == 5:
+                k[0] = 6.0                                 # the heavy hitter: visual token 6, in the mid region
+            q = np.array([1.0, 0.0, 0.0, 0.0]) if i < (cfg.budget_lines - 1) * n else np.array([-1.0, 1.0, 0.0, 0.0])
+            u.step(q[None, :], k, np.zeros(4))
+            if (i + 1) % n == 0 and (i + 1) < cfg.budget_lines * n:
+                assert u.line_end() is None
+        res = u.line_end()
+        kept[sn] = 5 not in set(int(p) for p in res["evicted_pos"])
+    assert kept[2] and not kept[0]
