@@ -601,8 +601,9 @@ def main():
     ap.add_argument("--no-pdl", action="store_true")
     ap.add_argument("--per-layer-line-end", action="store_true", help="one line-end launch per layer instead of one for all layers")
     ap.add_argument("--tile-ranges", action="store_true", help="deal 32-row tiles, not whole units, to the decode CTAs")
-    ap.add_argument("--score-norm", default="mid", choices=["mid", "cache"],
-                    help="softmax of Eq. 9 over the mid keys (as written) or over the whole live cache (variant)")
+    ap.add_argument("--score-norm", default="mid", choices=["mid", "cache", "accum"],
+                    help="line-end scoring: Eq. 9 over the mid keys (as written), over the whole live cache (variant), or "
+                         "attention accumulated over all decode steps (the paper's 'w. AttAcc' ablation)")
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -75,6 +75,15 @@ typedef enum { LAR_BF16 = 0, LAR_FP32 = 1 } lar_dtype_t;
                                         the G heads.  The line-end kernel stages C + B keys in shared memory:
                                         configurations where they do not fit are rejected at creation. */
 
+#define LAR_FLAG_SCORE_ACCUM 0x40u   /* scoring of the paper's ablation "w. AttAcc" (Sec. 4.4, Table 6; the accumulated-attention
+                                        rule of the H2O-style baselines of Sec. 4.2): a cached token's score is the attention
+                                        probability Eq. 2-3 gave it, summed over every decode step since it was appended and
+                                        over the G heads, divided by n G.  Every line end (also below budget) adds the line's
+                                        sums -- the cache-normalised form of Eq. 9 over all live entries -- to one float per
+                                        slot in the slab; a compressing line end ranks the mid entries by that sum, and an
+                                        entry keeps its sum when the compaction moves it.  Needs the C + B live keys in shared
+                                        memory, as LAR_FLAG_SCORE_CACHE_NORM does (which it implies). */
+
 #define LAR_FLAG_HOST_DEFER_OUT 0x20u /* lar_decode_step_host does not make `stream` wait for its copy-out: the
                                         copy-out of a call then overlaps the kernels of the next calls as well.
                                         `out_host` of a call is complete only after lar_cache_host_join (or four

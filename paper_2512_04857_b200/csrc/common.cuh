@@ -26,6 +26,7 @@ struct LayerView {
     UnitState* state;       // [units]
     char* guide;            // [units][n][G][d] elements
     float* scores;          // [units][mid_pad]
+    float* acc;             // [units][cap_pad] attention mass accumulated per slot (accumulated-attention scoring only)
     unsigned* status;       // one word per cache
     int pages_per_unit, page_tokens, cap, cap_pad, mid_pad;
     int cond_len, line_width, budget_tokens, anchor_len, recent_lines, compressing;
@@ -35,7 +36,7 @@ struct LayerView {
 
 // Byte distance between the same array of consecutive layers (a kernel whose grid spans several layers).
 struct LayerStrides {
-    size_t pool, page_table, index_map, state, guide, scores;
+    size_t pool, page_table, index_map, state, guide, scores, acc;
 };
 __host__ __device__ inline LayerView layer_view_at(LayerView lv, const LayerStrides& ls, int layers_ahead) {
     const size_t y = (size_t)layers_ahead;
@@ -46,6 +47,7 @@ __host__ __device__ inline LayerView layer_view_at(LayerView lv, const LayerStri
     lv.state = reinterpret_cast<UnitState*>(reinterpret_cast<char*>(lv.state) + y * ls.state);
     lv.guide += y * ls.guide;
     lv.scores = reinterpret_cast<float*>(reinterpret_cast<char*>(lv.scores) + y * ls.scores);
+    if (lv.acc) lv.acc = reinterpret_cast<float*>(reinterpret_cast<char*>(lv.acc) + y * ls.acc);
     return lv;
 }
 

@@ -46,6 +46,7 @@ struct Layout {
     size_t off_imap, stride_imap;
     size_t off_guide, stride_guide;
     size_t off_scores, stride_scores;
+    size_t off_acc, stride_acc;  // accumulated attention per slot (LAR_FLAG_SCORE_ACCUM only, else empty)
     size_t off_kpool, off_vpool, stride_pool;
     size_t off_partials, off_tickets, tickets_bytes;  // decode scratch (shared by the layers)
     size_t staging_q, staging_k, staging_v, staging_o;  // offsets inside one staging slot
@@ -143,7 +144,7 @@ bool derive(const lar_config_t* c, Derived& d) {
     // A unit of T tiles is cut into at most ceil(T / floor(U T / P)) + 1 segments (never more than T or P).
     // line end: one CTA per unit, 8 warps; few units with a large mid region get one warp per 16 guide rows (16..32 warps)
     d.le_threads = 256;
-    if (d.units <= 2 * kDefaultDecodeCtas && d.M >= 128) {
+    if ((c->flags & LAR_FLAG_SCORE_ACCUM) == 0 && d.units <= 2 * kDefaultDecodeCtas && d.M >= 128) {  // (accumulated attention: a column sum per warp over every live row -- 8 warps keep that in shared memory)
         const int blocks = (c->line_width * d.group + 15) / 16;
         d.le_threads = 32 * (blocks < 16 ? 16 : blocks > 32 ? 32 : blocks);
     }
@@ -182,6 +183,8 @@ void make_layout(const lar_config_t* c, const Derived& d, Layout& L) {
     L.off_guide = take(L.stride_guide * Lyr);
     L.stride_scores = align_up(U * d.mid_pad * 4, 256);
     L.off_scores = take(L.stride_scores * Lyr);
+    L.stride_acc = (c->flags & LAR_FLAG_SCORE_ACCUM) ? align_up(U * d.cap_pad * 4, 256) : 0;
+    L.off_acc = take(L.stride_acc * Lyr);
     L.stride_pool = align_up(U * d.ppu * d.P * d.row_bytes, 256);
     L.off_kpool = take(L.stride_pool * Lyr);
     L.off_vpool = take(L.stride_pool * Lyr);
@@ -254,7 +257,8 @@ lar_status_t plan_query_impl(const lar_config_t* cfg, lar_plan_t* out, Derived* 
     p.line_end_smem_bytes =
         d.compressing ? lar::line_end_smem_bytes(d.row_bytes, cfg->head_dim, d.M, d.M - cfg->line_width + cfg->recent_lines * cfg->line_width, d.le_threads / 32,
                                                  cfg->line_width * d.group, cfg->dtype == LAR_BF16 ? 1 : 0, cfg->cond_len + d.B,
-                                                 (cfg->flags & LAR_FLAG_SCORE_CACHE_NORM) ? 1 : 0) : 0;
+                                                 (cfg->flags & (LAR_FLAG_SCORE_CACHE_NORM | LAR_FLAG_SCORE_ACCUM)) ? 1 : 0,
+                                                 (cfg->flags & LAR_FLAG_SCORE_ACCUM) ? 1 : 0) : 0;
     p.slab_bytes = L.total;
     p.scratch_bytes = (L.off_tickets + L.tickets_bytes) - L.off_partials;
     if (p.decode_smem_bytes > 227 * 1024 || p.line_end_smem_bytes > 227 * 1024) return LAR_ERR_INVALID_ARG;
@@ -324,6 +328,7 @@ lar::LayerView view_of(const lar_cache* c, int layer) {
     v.state = reinterpret_cast<lar::UnitState*>(c->slab + L.off_state + L.stride_state * layer);
     v.guide = c->slab + L.off_guide + L.stride_guide * layer;
     v.scores = reinterpret_cast<float*>(c->slab + L.off_scores + L.stride_scores * layer);
+    v.acc = L.stride_acc ? reinterpret_cast<float*>(c->slab + L.off_acc + L.stride_acc * layer) : nullptr;
     v.status = reinterpret_cast<unsigned*>(c->slab + L.off_status);
     v.pages_per_unit = d.ppu;
     v.page_tokens = d.P;
@@ -631,6 +636,7 @@ lar_status_t lar_cache_create(const lar_config_t* cfg, void* dev_slab, size_t sl
     if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_state, 0, L.stride_state * cfg->n_layers);
     if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_imap, 0xff, L.stride_imap * cfg->n_layers);
     if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_scores, 0, L.stride_scores * cfg->n_layers);
+    if (ce == cudaSuccess && L.stride_acc) ce = cudaMemset(c->slab + L.off_acc, 0, L.stride_acc * cfg->n_layers);
     if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_guide, 0, L.stride_guide * cfg->n_layers);
     // rows of a page beyond the live length are read by short tiles with weight 0: they must be finite
     if (ce == cudaSuccess) ce = cudaMemset(c->slab + L.off_kpool, 0, L.stride_pool * cfg->n_layers);
@@ -670,6 +676,8 @@ lar_status_t lar_cache_reset(lar_cache_t* c, void* stream) {
     if (!c) return LAR_ERR_INVALID_ARG;
     LAR_CUDA(cudaMemsetAsync(c->slab + c->L.off_state, 0, c->L.stride_state * c->cfg.n_layers, (cudaStream_t)stream));
     LAR_CUDA(cudaMemsetAsync(c->slab + c->L.off_tickets, 0, c->L.tickets_bytes, (cudaStream_t)stream));
+    if (c->L.stride_acc)  // accumulated attention restarts with the image
+        LAR_CUDA(cudaMemsetAsync(c->slab + c->L.off_acc, 0, c->L.stride_acc * c->cfg.n_layers, (cudaStream_t)stream));
     LAR_CUDA(cudaMemsetAsync(c->slab + c->L.off_status + 128, 0, sizeof(int), (cudaStream_t)stream));
     for (auto& s : c->sh) s = LayerShadow();
     c->last_layer = -1;
@@ -842,6 +850,11 @@ lar_status_t lar_cache_host_join(lar_cache_t* c, void* stream) {
     return LAR_OK;
 }
 
+// scoring mode of the line-end kernel: bit 0 softmax over the whole live cache, bit 1 accumulated attention
+static int line_end_mode(const lar_cache* c) {
+    return ((c->cfg.flags & LAR_FLAG_SCORE_CACHE_NORM) ? 1 : 0) | ((c->cfg.flags & LAR_FLAG_SCORE_ACCUM) ? 2 : 0);
+}
+
 static lar::LayerStrides layer_strides(const lar_cache* c) {
     lar::LayerStrides ls;
     ls.pool = c->L.stride_pool;
@@ -850,6 +863,7 @@ static lar::LayerStrides layer_strides(const lar_cache* c) {
     ls.state = c->L.stride_state;
     ls.guide = c->L.stride_guide;
     ls.scores = c->L.stride_scores;
+    ls.acc = c->L.stride_acc;
     return ls;
 }
 
@@ -863,7 +877,7 @@ lar_status_t lar_line_end_score_evict(lar_cache_t* c, int layer, void* stream) {
         const lar::LayerView lv = view_of(c, layer);
         LineEndFn fn = line_end_fn(c->cfg, c->d.group);
         fn<<<dim3((unsigned)c->d.units, 1, 1), c->d.le_threads, c->plan.line_end_smem_bytes, (cudaStream_t)stream>>>(
-            lv, layer_strides(c), c->scale * 1.4426950408889634f, (c->cfg.flags & LAR_FLAG_SCORE_CACHE_NORM) ? 1 : 0);
+            lv, layer_strides(c), c->scale * 1.4426950408889634f, line_end_mode(c));
         LAR_CUDA(cudaGetLastError());
         c->launches++;
         c->last_layer = -2;  // rows of the cache were just moved: the next decode launch must not fetch ahead
@@ -884,7 +898,7 @@ lar_status_t lar_line_end_score_evict_all(lar_cache_t* c, void* stream) {
         LineEndFn fn = line_end_fn(c->cfg, c->d.group);
         fn<<<dim3((unsigned)c->d.units, (unsigned)c->cfg.n_layers, 1), c->d.le_threads, c->plan.line_end_smem_bytes,
              (cudaStream_t)stream>>>(lv, layer_strides(c), c->scale * 1.4426950408889634f,
-                                     (c->cfg.flags & LAR_FLAG_SCORE_CACHE_NORM) ? 1 : 0);
+                                     line_end_mode(c));
         LAR_CUDA(cudaGetLastError());
         c->launches++;
         c->last_layer = -2;  // every layer's cache was just written: the next decode launch must not fetch ahead

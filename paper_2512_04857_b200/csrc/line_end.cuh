@@ -50,13 +50,16 @@ __global__ void __launch_bounds__(128) append_kernel(const LayerView lv, const T
 __host__ __device__ inline int line_end_staged_rows(int M, int live_rows, int cache_norm) {
     return cache_norm ? (live_rows + 7) / 8 * 8 + 8 : (M + 7) / 8 * 8;
 }
+// accum (attention accumulated over all history; implies cache_norm): the column sums cover every live row, not only
+// the mid ones.
 __host__ __device__ inline int line_end_smem_bytes(int row_bytes, int D, int M, int total_rows, int warps, int nq, int is_bf16,
-                                                   int live_rows, int cache_norm) {
+                                                   int live_rows, int cache_norm, int accum) {
+    const int cols = accum ? live_rows : M;  // columns whose probabilities are summed
     int b = line_end_staged_rows(M, live_rows, cache_norm) * (row_bytes + 16);  // keys, rows padded by one chunk against bank conflicts
     if (is_bf16)
-        b += (cache_norm ? 0 : ((nq + 15) / 16 * 16) * (row_bytes + 16)) + warps * M * 4;  // guide rows (whole 16-row tiles), column sums per warp
+        b += (cache_norm ? 0 : ((nq + 15) / 16 * 16) * (row_bytes + 16)) + warps * cols * 4;  // guide rows (whole 16-row tiles), column sums per warp
     else
-        b += warps * (D + (cache_norm ? live_rows : M) + M) * 4;  // per warp: query row (fp32), logits row, score accumulator
+        b += warps * (D + (cache_norm ? live_rows : M) + cols) * 4;  // per warp: query row (fp32), logits row, score accumulator
     b += M * 4;                            // final scores
     b += ((M + 3) / 4) * 4;                // keep flags
     b += total_rows * 4;                   // source slot of every surviving row
@@ -148,18 +151,20 @@ __device__ __forceinline__ void score_mma(const unsigned char* keys, const unsig
         for (int k0 = 0; k0 < M; k0 += 8) {
             float c[4];
             logits(mid_off + k0, c);
-            float v0 = (w0 != 0.f ? exp2f(c[0] - m0) * w0 : 0.f) + (w1 != 0.f ? exp2f(c[2] - m1) * w1 : 0.f);
-            float v1 = (w0 != 0.f ? exp2f(c[1] - m0) * w0 : 0.f) + (w1 != 0.f ? exp2f(c[3] - m1) * w1 : 0.f);
+            // (a column may be a token of the line itself: a row gives it mass only if it was live for that row)
+            const int key = mid_off + k0 + 2 * quad;
+            float v0 = (w0 != 0.f && key < lim0 ? exp2f(c[0] - m0) * w0 : 0.f) + (w1 != 0.f && key < lim1 ? exp2f(c[2] - m1) * w1 : 0.f);
+            float v1 = (w0 != 0.f && key + 1 < lim0 ? exp2f(c[1] - m0) * w0 : 0.f) + (w1 != 0.f && key + 1 < lim1 ? exp2f(c[3] - m1) * w1 : 0.f);
 #pragma unroll
             for (int off = 4; off <= 16; off <<= 1) {
                 v0 += __shfl_xor_sync(0xffffffffu, v0, off);
                 v1 += __shfl_xor_sync(0xffffffffu, v1, off);
             }
             if (grow == 0) {  // lanes 0..3 own two keys each of this tile in the warp's row of column sums
-                const int key = k0 + 2 * quad;
+                const int col = k0 + 2 * quad;
                 float* mine = colsum + warp * M;
-                if (key < M) mine[key] += v0;
-                if (key + 1 < M) mine[key + 1] += v1;
+                if (col < M) mine[col] += v0;
+                if (col + 1 < M) mine[col + 1] += v1;
             }
         }
     }
@@ -170,7 +175,7 @@ __device__ __forceinline__ void score_mma(const unsigned char* keys, const unsig
 // (every guide query over the entries that were live when it was decoded).  Scoring: bf16 on tensor cores (score_mma); fp32 on CUDA cores, where every lane owns the keys
 // m = lane, lane + 32, ... and computes whole dot products against a query row broadcast from shared memory.
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, const LayerStrides ls, float scale_log2, int cache_norm) {
+__global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, const LayerStrides ls, float scale_log2, int mode) {
     constexpr int EPL = Elt<T>::kPerChunk;
     constexpr int ROW_BYTES = D * (int)sizeof(T);
     constexpr int CHUNKS = ROW_BYTES / 16;
@@ -188,7 +193,12 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
         if (tid == 0) atomicOr(lv.status, kStBoundary);
         return;
     }
-    if (v < B) return;  // cache below budget: nothing to evict (the queue restarts by itself)
+    // mode bit 0: softmax of Eq. 9 over the whole live cache; bit 1: rank by the attention accumulated over all decode
+    // steps (the per-line sums of the cache-normalised form, added up line by line in lv.acc)
+    const bool accum = (mode & 2) != 0;
+    const int cache_norm = (mode & 1) | (accum ? 1 : 0);
+    const bool compress = v == B;
+    if (!compress && !accum) return;  // cache below budget: nothing to evict (the queue restarts by itself)
 
     const int mid0 = C + lv.anchor_len;                       // first mid slot
     const int M = B - lv.anchor_len - lv.recent_lines * n;    // mid entries
@@ -206,10 +216,12 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
     unsigned char* kst = smem;
     unsigned char* after_k = smem + (size_t)rows_pad * KROW;
     unsigned char* qg = after_k;                                                // [nq16][KROW]   (bf16, mid-only scoring)
-    float* colsum = reinterpret_cast<float*>(after_k + (cache_norm ? (size_t)0 : (size_t)nq16 * KROW));  // [W][M] (bf16)
-    const int wstride = D + n_stage + M;
-    float* wbuf = reinterpret_cast<float*>(after_k);                            // [W][D + n_stage + M]   (fp32)
-    float* S = kMma ? colsum + W * M : wbuf + W * wstride;
+    // columns whose probabilities are summed: the M mid keys, or (accum) every staged row
+    const int cols = accum ? n_stage : M, col_off = accum ? 0 : mid_off;
+    float* colsum = reinterpret_cast<float*>(after_k + (cache_norm ? (size_t)0 : (size_t)nq16 * KROW));  // [W][cols] (bf16)
+    const int wstride = D + n_stage + cols;
+    float* wbuf = reinterpret_cast<float*>(after_k);                            // [W][D + n_stage + cols]   (fp32)
+    float* S = kMma ? colsum + W * cols : wbuf + W * wstride;
     unsigned char* keep = reinterpret_cast<unsigned char*>(S + M);
     int* srcmap = reinterpret_cast<int*>(keep + ((M + 3) / 4) * 4);
 
@@ -231,21 +243,12 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
                 *reinterpret_cast<uint4*>(qg + r * KROW + c * 16) = val;
             }
         }
-        for (int mm = tid; mm < W * M; mm += blockDim.x) colsum[mm] = 0.f;
+        for (int mm = tid; mm < W * cols; mm += blockDim.x) colsum[mm] = 0.f;
         __syncthreads();
         if (cache_norm)
-            score_mma<D, true>(kst, qg, reinterpret_cast<const uint32_t*>(gq), colsum, n_stage, mid_off, M, nq, G, n, scale_log2, warp, lane, W);
+            score_mma<D, true>(kst, qg, reinterpret_cast<const uint32_t*>(gq), colsum, n_stage, col_off, cols, nq, G, n, scale_log2, warp, lane, W);
         else
-            score_mma<D, false>(kst, qg, nullptr, colsum, n_stage, mid_off, M, nq, G, n, scale_log2, warp, lane, W);
-        __syncthreads();
-        const float inv_nq = 1.f / (float)nq;
-        for (int mm = tid; mm < M; mm += blockDim.x) {
-            float sc = 0.f;
-            for (int w = 0; w < W; ++w) sc += colsum[w * M + mm];
-            sc *= inv_nq;
-            S[mm] = sc;
-            lv.scores[(size_t)unit * lv.mid_pad + mm] = sc;
-        }
+            score_mma<D, false>(kst, qg, nullptr, colsum, n_stage, col_off, cols, nq, G, n, scale_log2, warp, lane, W);
         __syncthreads();
     } else {
         // ---- Eq. 9 on CUDA cores: every guide row is soft-maxed over its keys (the M mid keys, or the entries that
@@ -253,7 +256,7 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
         float* qrow = wbuf + warp * wstride;
         float* logit = qrow + D;
         float* sacc = logit + n_stage;
-        for (int mm = lane; mm < M; mm += 32) sacc[mm] = 0.f;
+        for (int mm = lane; mm < cols; mm += 32) sacc[mm] = 0.f;
         __syncthreads();
         for (int j = warp; j < nq; j += W) {
             for (int c = lane; c < CHUNKS; c += 32) {
@@ -289,20 +292,43 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
             sum = warp_sum(sum);
             const float inv = 1.f / sum;
             __syncwarp();
-            for (int mm = lane; mm < M; mm += 32) sacc[mm] = fmaf(logit[mid_off + mm], inv, sacc[mm]);
+            for (int mm = lane; mm < cols && col_off + mm < lim; mm += 32) sacc[mm] = fmaf(logit[col_off + mm], inv, sacc[mm]);
             __syncwarp();
         }
         __syncthreads();
+    }
+    // ---- the line's score of every column: the warps' sums added in a fixed order (reproducible kept sets)
+    {
+        const float* wsum = kMma ? colsum : wbuf + D + n_stage;
+        const int wsum_stride = kMma ? cols : wstride;
         const float inv_nq = 1.f / (float)nq;
-        for (int mm = tid; mm < M; mm += blockDim.x) {
-            float sc = 0.f;
-            for (int w = 0; w < W; ++w) sc += wbuf[w * wstride + D + n_stage + mm];
-            sc *= inv_nq;
-            S[mm] = sc;
-            lv.scores[(size_t)unit * lv.mid_pad + mm] = sc;
+        if (!accum) {
+            for (int mm = tid; mm < M; mm += blockDim.x) {
+                float sc = 0.f;
+                for (int w = 0; w < W; ++w) sc += wsum[w * wsum_stride + mm];
+                sc *= inv_nq;
+                S[mm] = sc;
+                lv.scores[(size_t)unit * lv.mid_pad + mm] = sc;
+            }
+        } else {
+            // every live slot adds the line's mass to what it had; the line's own tokens (the last n slots) start here
+            float* acc = lv.acc + (size_t)unit * lv.cap_pad;
+            for (int sl = tid; sl < n_stage; sl += blockDim.x) {
+                float sc = 0.f;
+                for (int w = 0; w < W; ++w) sc += wsum[w * wsum_stride + sl];
+                sc *= inv_nq;
+                const float total = (sl >= n_stage - n ? 0.f : acc[sl]) + sc;
+                acc[sl] = total;
+                const int mm = sl - mid0;
+                if (compress && mm >= 0 && mm < M) {
+                    S[mm] = total;
+                    lv.scores[(size_t)unit * lv.mid_pad + mm] = total;
+                }
+            }
         }
         __syncthreads();
     }
+    if (!compress) return;  // (accumulated-attention scoring below budget: the sums are updated, nothing is evicted)
 
     // ---- Eq. 10: keep the M - n most salient; equal scores keep the lower slot (older token).
     // A score that is not finite (a NaN or Inf in a key or query) has no rank: it is treated as the lowest possible
@@ -349,6 +375,7 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
         const int rows = min(tile_rows, total_rows - t0);
         uint4 kbuf[PER_THREAD], vbuf[PER_THREAD];
         int ibuf = 0;
+        float abuf = 0.f;
 #pragma unroll
         for (int i = 0; i < PER_THREAD; ++i) {
             const int idx = tid + i * nthr;
@@ -362,7 +389,10 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
                 }
             }
         }
-        if (tid < rows) ibuf = imap[mid0 + srcmap[t0 + tid]];
+        if (tid < rows) {
+            ibuf = imap[mid0 + srcmap[t0 + tid]];
+            if (accum) abuf = lv.acc[(size_t)unit * lv.cap_pad + mid0 + srcmap[t0 + tid]];
+        }
         __syncthreads();
 #pragma unroll
         for (int i = 0; i < PER_THREAD; ++i) {
@@ -376,7 +406,10 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
                 }
             }
         }
-        if (tid < rows) imap[mid0 + t0 + tid] = ibuf;
+        if (tid < rows) {
+            imap[mid0 + t0 + tid] = ibuf;
+            if (accum) lv.acc[(size_t)unit * lv.cap_pad + mid0 + t0 + tid] = abuf;
+        }
         __syncthreads();
     }
     if (tid == 0) {

@@ -19,6 +19,7 @@ LAR_BF16, LAR_FP32 = 0, 1
 LAR_FLAG_NO_HOST_CHECKS, LAR_FLAG_PDL, LAR_FLAG_SHUFFLE_PAGES, LAR_FLAG_TILE_RANGES = 0x1, 0x2, 0x4, 0x8
 LAR_FLAG_SCORE_CACHE_NORM = 0x10
 LAR_FLAG_HOST_DEFER_OUT = 0x20
+LAR_FLAG_SCORE_ACCUM = 0x40
 
 
 class lar_config_t(C.Structure):
@@ -107,6 +108,8 @@ def config_from_workload(w, **overrides) -> lar_config_t:
     kw.update(overrides)
     if getattr(w, "score_norm", "mid") == "cache":
         kw["flags"] = kw.get("flags", 0) | LAR_FLAG_SCORE_CACHE_NORM
+    if getattr(w, "score_norm", "mid") == "accum":
+        kw["flags"] = kw.get("flags", 0) | LAR_FLAG_SCORE_ACCUM
     return make_config(**kw)
 
 

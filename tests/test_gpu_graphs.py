@@ -26,7 +26,7 @@ def _args(**kw):
     ("janus_pro_7b", dict(n_layers=3, batch=2, n_q_heads=4, n_kv_heads=4)),
     ("gqa_1024", dict(n_layers=2, batch=2, n_q_heads=8, n_kv_heads=2, n_lines=12)),
 ])
-@pytest.mark.parametrize("tile_ranges,score_norm", [(False, "mid"), (True, "mid"), (False, "cache")])
+@pytest.mark.parametrize("tile_ranges,score_norm", [(False, "mid"), (True, "mid"), (False, "cache"), (False, "accum")])
 def test_graph_replay_of_a_second_generation_matches_the_oracle(shape, kw, tile_ranges, score_norm):
     w = W.WORKLOADS[shape].scaled(score_norm=score_norm, **kw)
     dev = torch.device("cuda:0")

@@ -214,8 +214,11 @@ def test_generator_gpu_matches_cpu():
     dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=1),
     dict(dtype="bf16", head_dim=64, n_q_heads=4, n_kv_heads=4, cond_len=3, anchor_len=5, recent_lines=2, budget_lines=5),
 ])
-def test_cache_normalised_scoring(kw):
-    w = W.WORKLOADS["tiny_b"].scaled(score_norm="cache", **kw)
+@pytest.mark.parametrize("score_norm", ["cache", "accum"])
+def test_cache_normalised_scoring(kw, score_norm):
+    """The two scoring variants that soft-max over the whole live cache: the line's own decode probabilities ("cache"),
+    and those probabilities accumulated over every step since a token was appended ("accum", the paper's ablation)."""
+    w = W.WORKLOADS["tiny_b"].scaled(score_norm=score_norm, **kw)
     rep = run_parity(w)
     _check(rep, w, allow_near_ties=1)
     assert rep.compressions > 0
@@ -233,9 +236,19 @@ def test_cache_normalised_scoring_one_launch_for_all_layers():
     assert rep.max_score_rel_err < 1e-4
 
 
+def test_accumulated_attention_scoring_one_launch_for_all_layers_and_unfused_appends():
+    w = W.WORKLOADS["tiny_b"].scaled(score_norm="accum", n_layers=3, dtype="bf16", n_q_heads=4, n_kv_heads=2)
+    assert lar.config_from_workload(w).flags & lar.LAR_FLAG_SCORE_ACCUM
+    for fused in (True, False):
+        rep = run_parity(w, line_end_all=True, fused=fused)
+        _check(rep, w, allow_near_ties=1)
+        assert rep.compressions > 0 and rep.max_score_rel_err < 2e-3
+
+
+@pytest.mark.parametrize("score_norm", ["cache", "accum"])
 @pytest.mark.parametrize("name,layers,n_units", [("janus_pro_7b", 2, 4), ("gqa_1024", 1, 3)])
-def test_cache_normalised_scoring_full_size_sampled(name, layers, n_units):
-    w = W.WORKLOADS[name].scaled(n_layers=layers, score_norm="cache")
+def test_cache_normalised_scoring_full_size_sampled(name, layers, n_units, score_norm):
+    w = W.WORKLOADS[name].scaled(n_layers=layers, score_norm=score_norm)
     rep = run_parity(w, units=pick_units(w, n_units, seed=3), gen_device="cuda", cfg_overrides=dict(flags=lar.LAR_FLAG_PDL),
                      line_end_all=True)
     _check(rep, w, allow_near_ties=2)
