@@ -207,6 +207,8 @@ class Runner:
             flags |= lar.LAR_FLAG_PDL
         if args.tile_ranges:
             flags |= lar.LAR_FLAG_TILE_RANGES
+        if getattr(args, "slot_reuse", False):
+            flags |= lar.LAR_FLAG_SLOT_REUSE
         self.cfg = lar.config_from_workload(w, flags=flags, kv_splits=args.kv_splits, warps_per_cta=args.warps,
                                             stages=args.stages, page_tokens=args.page_tokens, decode_ctas=args.ctas)
         self.cache = lar.Cache(self.cfg, device=str(dev))
@@ -480,7 +482,8 @@ def run_ours(args):
                        "budget_lines": w.budget_lines, "anchor": w.anchor_len, "recent_lines": w.recent_lines,
                        "score_norm": w.score_norm,
                        "launch": ("cuda-graph per line, fused append+decode" + (", PDL" if not args.no_pdl else "") +
-                                  (", line end per layer" if args.per_layer_line_end else ", one line-end launch for all layers")),
+                                  (", line end per layer" if args.per_layer_line_end else ", one line-end launch for all layers") +
+                                  (", slot reuse instead of compaction" if args.slot_reuse else "")),
                        "l2": "inputs larger than L2: all layers cycled every token "
                              f"({kv_bytes / n_decode / 1e6:.0f} MB per launch x {w.n_layers} layers)",
                        "plan": main["plan"], "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
@@ -604,6 +607,8 @@ def main():
     ap.add_argument("--score-norm", default="mid", choices=["mid", "cache", "accum"],
                     help="line-end scoring: Eq. 9 over the mid keys (as written), over the whole live cache (variant), or "
                          "attention accumulated over all decode steps (the paper's 'w. AttAcc' ablation)")
+    ap.add_argument("--slot-reuse", action="store_true",
+                    help="line end without compaction: the evicted slots take the newest line's rows (LAR_FLAG_SLOT_REUSE)")
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -84,6 +84,13 @@ typedef enum { LAR_BF16 = 0, LAR_FP32 = 1 } lar_dtype_t;
                                         entry keeps its sum when the compaction moves it.  Needs the C + B live keys in shared
                                         memory, as LAR_FLAG_SCORE_CACHE_NORM does (which it implies). */
 
+#define LAR_FLAG_SLOT_REUSE 0x80u    /* the line end does not compact (Eq. 5-7 define the kept SET; Eq. 2 does not depend on
+                                        the order of the cache): the n evicted slots take the n rows of the newest line, so
+                                        n rows of K and V move instead of every row behind the first hole, and the cache
+                                        stays dense for the decode kernel.  Slots then no longer follow original positions
+                                        (the index map is not monotone); the line end finds the mid region of Sec. 3.3
+                                        through the index map.  Kept sets, outputs and scores are unchanged. */
+
 #define LAR_FLAG_HOST_DEFER_OUT 0x20u /* lar_decode_step_host does not make `stream` wait for its copy-out: the
                                         copy-out of a call then overlaps the kernels of the next calls as well.
                                         `out_host` of a call is complete only after lar_cache_host_join (or four
@@ -174,6 +181,18 @@ lar_status_t lar_decode_attn(lar_cache_t* c, int layer, const void* q, void* out
  * k, v: device, [batch, n_kv_heads, head_dim], 16-byte aligned. */
 lar_status_t lar_decode_step(lar_cache_t* c, int layer, const void* q, const void* k, const void* v,
                              void* out, void* stream);
+
+/* lar_decode_step on views of larger tensors (bf16 storage only): consecutive sequences of q, k, v, out lie
+ * *_seq_stride ELEMENTS apart, the heads of one sequence back to back -- e.g. q, k and v as column ranges of the
+ * [batch, (n_q_heads + 2 n_kv_heads) * head_dim] output of a fused QKV projection (the three strides are then that row
+ * length), and out as a view of the buffer the output projection reads.  The cache therefore takes the keys exactly as
+ * the caller hands them over: a model with rotary position embedding passes post-rotation k and q, so that the guide
+ * queries of Eq. 8 and the cached keys of Eq. 9 live in the same space (Sec. 3.3).
+ * Every stride is a multiple of 8 elements (16 bytes) and at least the dense row of its tensor, every pointer 16-byte
+ * aligned; otherwise LAR_ERR_INVALID_ARG (also for fp32 caches).  Call order and errors as lar_decode_step. */
+lar_status_t lar_decode_step_strided(lar_cache_t* c, int layer, const void* q, const void* k, const void* v, void* out,
+                                     int64_t q_seq_stride, int64_t k_seq_stride, int64_t v_seq_stride,
+                                     int64_t out_seq_stride, void* stream);
 
 /* lar_decode_step with HOST buffers (pinned memory): copies q, k, v to a staging area of the slab, runs the
  * fused kernel and copies `out` back, asynchronously.  Seen from `stream` the call is one stream-ordered

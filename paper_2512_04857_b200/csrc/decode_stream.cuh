@@ -66,6 +66,9 @@ struct StreamArgs {
     int* done_seq;      // device word: every launch up to this number has completed
     int q_slots, p_bufs;  // depth of the CTA's query ring / number of partial buffers
     int pool_row_base;  // first pool row of this layer in the tensor maps
+    // elements between consecutive sequences of q / k_new / v_new / out (0: dense, heads of a sequence back to back and
+    // sequences back to back); within a sequence the heads are always back to back
+    long long q_seq_stride, k_seq_stride, v_seq_stride, out_seq_stride;
 };
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar, uint64_t policy) {
@@ -281,6 +284,12 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     // One lane requests the inputs of segment `seg`: its queries and, where the segment closes its unit in a fused
     // step, the new k and v rows.  Issued by the epilogue warp, which is idle when a launch starts, so that the
     // producer's first K/V copies are not queued behind them.
+    // element offset of unit `u`'s rows in a [sequence][head][d] tensor with `per_head` elements per KV head
+    auto unit_offset = [&](int u, long long seq_stride, int per_head) -> size_t {
+        if (seq_stride == 0) return (size_t)u * per_head;
+        const int sq = u / lv.n_kv_heads;
+        return (size_t)sq * (size_t)seq_stride + (size_t)(u - sq * lv.n_kv_heads) * per_head;
+    };
     auto issue_inputs = [&](int seg) -> bool {
         const int slot = seg % NQ;
         if (seg >= NQ && !wait_or_abort(bar_qempty + slot * 8, (uint32_t)((seg / NQ - 1) & 1), abort_flag)) return false;
@@ -289,10 +298,10 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         const bool with_kv = a.fused && closes;
         const uint32_t bar = bar_qfull + slot * 8, dst = qring + slot * QENT;
         mbar_expect_tx(bar, (uint32_t)((G + (with_kv ? 2 : 0)) * D * 2));
-        bulk_g2s(dst, reinterpret_cast<const T16*>(a.q) + (size_t)unit * G * D, G * D * 2, bar);
+        bulk_g2s(dst, reinterpret_cast<const T16*>(a.q) + unit_offset(unit, a.q_seq_stride, G * D), G * D * 2, bar);
         if (with_kv) {
-            bulk_g2s(dst + G * D * 2, reinterpret_cast<const T16*>(a.k_new) + (size_t)unit * D, D * 2, bar);
-            bulk_g2s(dst + (G + 1) * D * 2, reinterpret_cast<const T16*>(a.v_new) + (size_t)unit * D, D * 2, bar);
+            bulk_g2s(dst + G * D * 2, reinterpret_cast<const T16*>(a.k_new) + unit_offset(unit, a.k_seq_stride, D), D * 2, bar);
+            bulk_g2s(dst + (G + 1) * D * 2, reinterpret_cast<const T16*>(a.v_new) + unit_offset(unit, a.v_seq_stride, D), D * 2, bar);
         }
         return true;
     };
@@ -583,6 +592,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             const int unit = u0 + seg;
             const int ub = unit * T;
             const bool opens = ub >= t_begin, closes = ub + T <= t_end;
+            const size_t out_base = unit_offset(unit, a.out_seq_stride, G * D);
             const int qs = seg % NQ, buf = seg % NPB;
             closing_loads(seg + 1, page_nxt, dev_len_nxt);
             ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag);
@@ -700,7 +710,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                 const float inv = Lh > 0.f ? 1.f / Lh : 0.f;
 #pragma unroll
                 for (int i = 0; i < EPH; ++i)
-                    outp[((size_t)unit * G + hg) * D + sub + LPH * i] = __float2bfloat16_rn(Oh[i] * inv);
+                    outp[out_base + (size_t)hg * D + sub + LPH * i] = __float2bfloat16_rn(Oh[i] * inv);
             } else {
                 // the unit is shared with neighbouring CTAs: leave a partial, the last one to arrive merges
                 const int p_first = range_owner(ub, total, Pe);
@@ -768,7 +778,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                             const float inv = L[c] > 0.f ? 1.f / L[c] : 0.f;
 #pragma unroll
                             for (int i = 0; i < PER; ++i)
-                                outp[((size_t)unit * G + g0 + c) * D + lane + 32 * i] = __float2bfloat16_rn(O[c][i] * inv);
+                                outp[out_base + (size_t)(g0 + c) * D + lane + 32 * i] = __float2bfloat16_rn(O[c][i] * inv);
                         }
                     }
                     if (lane == 0) a.tickets[unit] = 0;

@@ -144,7 +144,11 @@ bool derive(const lar_config_t* c, Derived& d) {
     // A unit of T tiles is cut into at most ceil(T / floor(U T / P)) + 1 segments (never more than T or P).
     // line end: one CTA per unit, 8 warps; few units with a large mid region get one warp per 16 guide rows (16..32 warps)
     d.le_threads = 256;
-    if ((c->flags & LAR_FLAG_SCORE_ACCUM) == 0 && d.units <= 2 * kDefaultDecodeCtas && d.M >= 128) {  // (accumulated attention: a column sum per warp over every live row -- 8 warps keep that in shared memory)
+    // (a column sum per warp over every live row -- accumulated attention, or the cache-normalised form without
+    // compaction -- stays at 8 warps so that it fits into shared memory)
+    const bool all_cols = (c->flags & LAR_FLAG_SCORE_ACCUM) ||
+                          ((c->flags & LAR_FLAG_SLOT_REUSE) && (c->flags & LAR_FLAG_SCORE_CACHE_NORM));
+    if (!all_cols && d.units <= 2 * kDefaultDecodeCtas && d.M >= 128) {
         const int blocks = (c->line_width * d.group + 15) / 16;
         d.le_threads = 32 * (blocks < 16 ? 16 : blocks > 32 ? 32 : blocks);
     }
@@ -258,7 +262,8 @@ lar_status_t plan_query_impl(const lar_config_t* cfg, lar_plan_t* out, Derived* 
         d.compressing ? lar::line_end_smem_bytes(d.row_bytes, cfg->head_dim, d.M, d.M - cfg->line_width + cfg->recent_lines * cfg->line_width, d.le_threads / 32,
                                                  cfg->line_width * d.group, cfg->dtype == LAR_BF16 ? 1 : 0, cfg->cond_len + d.B,
                                                  (cfg->flags & (LAR_FLAG_SCORE_CACHE_NORM | LAR_FLAG_SCORE_ACCUM)) ? 1 : 0,
-                                                 (cfg->flags & LAR_FLAG_SCORE_ACCUM) ? 1 : 0) : 0;
+                                                 (cfg->flags & LAR_FLAG_SCORE_ACCUM) ? 1 : 0,
+                                                 (cfg->flags & LAR_FLAG_SLOT_REUSE) ? 1 : 0, d.N) : 0;
     p.slab_bytes = L.total;
     p.scratch_bytes = (L.off_tickets + L.tickets_bytes) - L.off_partials;
     if (p.decode_smem_bytes > 227 * 1024 || p.line_end_smem_bytes > 227 * 1024) return LAR_ERR_INVALID_ARG;
@@ -448,8 +453,13 @@ lar_status_t launch_append(lar_cache* c, int layer, const void* k, const void* v
     return LAR_OK;
 }
 
+// Elements between consecutive sequences of q, k, v and out (0 = dense).
+struct SeqStrides {
+    long long q = 0, k = 0, v = 0, out = 0;
+};
+
 lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k, const void* v, void* out, int fused,
-                           cudaStream_t s) {
+                           cudaStream_t s, const SeqStrides& ss = SeqStrides()) {
     const bool pdl = (c->cfg.flags & LAR_FLAG_PDL) != 0;
     // With programmatic dependent launch a CTA moves in as soon as an SM is free, a few microseconds before the
     // preceding kernel is done.  It requests its first ring of cached K/V tiles then, so that arithmetic starts when
@@ -507,6 +517,10 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
         a.q_slots = c->d.q_slots;
         a.p_bufs = c->d.p_bufs;
         a.pool_row_base = layer * c->rows_per_layer;
+        a.q_seq_stride = ss.q;
+        a.k_seq_stride = ss.k;
+        a.v_seq_stride = ss.v;
+        a.out_seq_stride = ss.out;
         lc.gridDim = dim3((unsigned)c->d.ctas, 1, 1);
         lc.blockDim = dim3((unsigned)(32 * (c->plan.warps_per_cta + lar::kProducers + 1)), 1, 1);
         lc.attrs = attrs;
@@ -514,6 +528,7 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
         DecodeStreamFn fn = decode_stream_fn(c->cfg, c->d.group);
         LAR_CUDA(cudaLaunchKernelEx(&lc, fn, a, c->tmaps));
     } else {
+        if (ss.q || ss.k || ss.v || ss.out) return LAR_ERR_INVALID_ARG;  // fp32 storage: dense tensors only
         lar::DecodeArgs a;
         a.lv = view_of(c, layer);
         a.q = q;
@@ -755,6 +770,32 @@ lar_status_t lar_decode_step(lar_cache_t* c, int layer, const void* q, const voi
     return LAR_OK;
 }
 
+lar_status_t lar_decode_step_strided(lar_cache_t* c, int layer, const void* q, const void* k, const void* v, void* out,
+                                     int64_t q_seq_stride, int64_t k_seq_stride, int64_t v_seq_stride, int64_t out_seq_stride,
+                                     void* stream) {
+    if (bad_layer(c, layer) || !q || !k || !v || !out) return LAR_ERR_INVALID_ARG;
+    if (c->cfg.dtype != LAR_BF16) return LAR_ERR_INVALID_ARG;
+    const int64_t d = c->cfg.head_dim, hq = c->cfg.n_q_heads, hkv = c->cfg.n_kv_heads;
+    // a sequence's heads must fit between two sequences; bulk copies need 16-byte (8-element) aligned rows
+    if (q_seq_stride < hq * d || out_seq_stride < hq * d || k_seq_stride < hkv * d || v_seq_stride < hkv * d) return LAR_ERR_INVALID_ARG;
+    if ((q_seq_stride | k_seq_stride | v_seq_stride | out_seq_stride) & 7) return LAR_ERR_INVALID_ARG;
+    LayerShadow& sh = c->sh[layer];
+    lar_status_t st = check_visual_append(c, sh);
+    if (st != LAR_OK) return st;
+    SeqStrides ss;
+    // (a stride that equals the dense one is passed as 0: the kernel then needs no division per unit)
+    ss.q = q_seq_stride == hq * d ? 0 : q_seq_stride;
+    ss.k = k_seq_stride == hkv * d ? 0 : k_seq_stride;
+    ss.v = v_seq_stride == hkv * d ? 0 : v_seq_stride;
+    ss.out = out_seq_stride == hq * d ? 0 : out_seq_stride;
+    st = launch_decode(c, layer, q, k, v, out, 1, (cudaStream_t)stream, ss);
+    if (st != LAR_OK) return st;
+    sh.v += 1;
+    sh.n_tok += 1;
+    sh.line_fill += 1;
+    return LAR_OK;
+}
+
 // Host buffers in, host buffer out.  Three streams: the caller's (kernel), s_in (host -> device), s_out (device ->
 // host).  kHostSlots staging slots take turns, so the copy-in of call t + 1 overlaps the kernel and the copy-out of call t; the
 // caller's stream waits for the copy-out before the call returns its place in the stream, which keeps every effect of
@@ -852,7 +893,8 @@ lar_status_t lar_cache_host_join(lar_cache_t* c, void* stream) {
 
 // scoring mode of the line-end kernel: bit 0 softmax over the whole live cache, bit 1 accumulated attention
 static int line_end_mode(const lar_cache* c) {
-    return ((c->cfg.flags & LAR_FLAG_SCORE_CACHE_NORM) ? 1 : 0) | ((c->cfg.flags & LAR_FLAG_SCORE_ACCUM) ? 2 : 0);
+    return ((c->cfg.flags & LAR_FLAG_SCORE_CACHE_NORM) ? 1 : 0) | ((c->cfg.flags & LAR_FLAG_SCORE_ACCUM) ? 2 : 0) |
+           ((c->cfg.flags & LAR_FLAG_SLOT_REUSE) ? 4 : 0);
 }
 
 static lar::LayerStrides layer_strides(const lar_cache* c) {

@@ -52,9 +52,11 @@ __host__ __device__ inline int line_end_staged_rows(int M, int live_rows, int ca
 }
 // accum (attention accumulated over all history; implies cache_norm): the column sums cover every live row, not only
 // the mid ones.
+// reuse (the evicted slots are refilled, nothing is compacted): the mid entries are found through the index map; their
+// slots and a bitmap of the mid positions (n_visual bits, with word-wise prefix counts) are kept in shared memory as well.
 __host__ __device__ inline int line_end_smem_bytes(int row_bytes, int D, int M, int total_rows, int warps, int nq, int is_bf16,
-                                                   int live_rows, int cache_norm, int accum) {
-    const int cols = accum ? live_rows : M;  // columns whose probabilities are summed
+                                                   int live_rows, int cache_norm, int accum, int reuse, int n_visual) {
+    const int cols = (accum || (reuse && cache_norm)) ? live_rows : M;  // columns whose probabilities are summed
     int b = line_end_staged_rows(M, live_rows, cache_norm) * (row_bytes + 16);  // keys, rows padded by one chunk against bank conflicts
     if (is_bf16)
         b += (cache_norm ? 0 : ((nq + 15) / 16 * 16) * (row_bytes + 16)) + warps * cols * 4;  // guide rows (whole 16-row tiles), column sums per warp
@@ -63,6 +65,7 @@ __host__ __device__ inline int line_end_smem_bytes(int row_bytes, int D, int M, 
     b += M * 4;                            // final scores
     b += ((M + 3) / 4) * 4;                // keep flags
     b += total_rows * 4;                   // source slot of every surviving row
+    if (reuse) b += (M + 2 * ((n_visual + 31) / 32)) * 4;  // slots of the mid entries, bitmap of mid positions + prefix counts
     return (b + 15) / 16 * 16 + 16;
 }
 
@@ -195,7 +198,9 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
     }
     // mode bit 0: softmax of Eq. 9 over the whole live cache; bit 1: rank by the attention accumulated over all decode
     // steps (the per-line sums of the cache-normalised form, added up line by line in lv.acc)
-    const bool accum = (mode & 2) != 0;
+    // bit 2: no compaction -- the n evicted slots take the n rows of the newest line (n rows move instead of every row
+    // behind the first hole); slots then no longer follow positions, and the mid region is found through the index map
+    const bool accum = (mode & 2) != 0, reuse = (mode & 4) != 0;
     const int cache_norm = (mode & 1) | (accum ? 1 : 0);
     const bool compress = v == B;
     if (!compress && !accum) return;  // cache below budget: nothing to evict (the queue restarts by itself)
@@ -217,19 +222,66 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
     unsigned char* after_k = smem + (size_t)rows_pad * KROW;
     unsigned char* qg = after_k;                                                // [nq16][KROW]   (bf16, mid-only scoring)
     // columns whose probabilities are summed: the M mid keys, or (accum) every staged row
-    const int cols = accum ? n_stage : M, col_off = accum ? 0 : mid_off;
+    const bool all_cols = accum || (reuse && cache_norm);
+    const int cols = all_cols ? n_stage : M, col_off = all_cols ? 0 : mid_off;
     float* colsum = reinterpret_cast<float*>(after_k + (cache_norm ? (size_t)0 : (size_t)nq16 * KROW));  // [W][cols] (bf16)
     const int wstride = D + n_stage + cols;
     float* wbuf = reinterpret_cast<float*>(after_k);                            // [W][D + n_stage + cols]   (fp32)
     float* S = kMma ? colsum + W * cols : wbuf + W * wstride;
     unsigned char* keep = reinterpret_cast<unsigned char*>(S + M);
     int* srcmap = reinterpret_cast<int*>(keep + ((M + 3) / 4) * 4);
+    int* mid_slot = srcmap + total_rows;  // [M]   (reuse) slot of the mid entries, in ascending original position
+    unsigned* pos_bits = reinterpret_cast<unsigned*>(mid_slot + M);  // (reuse) bit p - lo_pos: a live entry has mid position p
+    int* imap = lv.index_map + (size_t)unit * lv.cap_pad;
+
+    if (reuse && compress) {
+        // ---- the mid region by position (Sec. 3.3): visual index in (N_init, (l - r) n].  The live mid positions are
+        // marked in a bitmap; an entry's place in ascending position is the number of marked bits below its own.
+        const int lo_pos = C + lv.anchor_len, hi_pos = C + (st.n_tok / n - lv.recent_lines) * n;  // mid: lo_pos <= pos < hi_pos
+        const int n_words = (hi_pos - lo_pos + 31) / 32;
+        int* below = reinterpret_cast<int*>(pos_bits + n_words);   // marked bits in the words before this one
+        for (int i = tid; i < n_words; i += blockDim.x) pos_bits[i] = 0u;
+        __syncthreads();
+        for (int sl = C + tid; sl < st.len; sl += blockDim.x) {
+            const int p = imap[sl];
+            if (p >= lo_pos && p < hi_pos) atomicOr(&pos_bits[(p - lo_pos) >> 5], 1u << ((p - lo_pos) & 31));
+        }
+        __syncthreads();
+        if (warp == 0) {
+            int run = 0;
+            for (int i0 = 0; i0 < n_words; i0 += 32) {
+                const int cnt = i0 + lane < n_words ? __popc(pos_bits[i0 + lane]) : 0;
+                int inc = cnt;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const int t = __shfl_up_sync(0xffffffffu, inc, off);
+                    if (lane >= off) inc += t;
+                }
+                if (i0 + lane < n_words) below[i0 + lane] = run + inc - cnt;
+                run += __shfl_sync(0xffffffffu, inc, 31);
+            }
+            if (lane == 0 && run != M) atomicOr(lv.status, kStBoundary);  // not exactly M mid entries: the index map is damaged
+        }
+        __syncthreads();
+        for (int sl = C + tid; sl < st.len; sl += blockDim.x) {
+            const int p = imap[sl];
+            if (p >= lo_pos && p < hi_pos) {
+                const int w = (p - lo_pos) >> 5, bit = (p - lo_pos) & 31;
+                const int rank = below[w] + __popc(pos_bits[w] & ((1u << bit) - 1u));
+                if (rank < M) mid_slot[rank] = sl;
+            }
+        }
+        __syncthreads();
+    }
 
     // ---- stage the keys (rows behind the last one are cleared)
     for (int idx = tid; idx < rows_pad * CHUNKS; idx += blockDim.x) {
         const int r = idx / CHUNKS, c = idx - r * CHUNKS;
         uint4 val = make_uint4(0u, 0u, 0u, 0u);
-        if (r < n_stage) val = *reinterpret_cast<const uint4*>(lv.k_pool + row_offset(lv, unit, stage0 + r, ROW_BYTES) + c * 16);
+        if (r < n_stage) {
+            const int sl = (reuse && !cache_norm) ? mid_slot[r] : stage0 + r;
+            val = *reinterpret_cast<const uint4*>(lv.k_pool + row_offset(lv, unit, sl, ROW_BYTES) + c * 16);
+        }
         *reinterpret_cast<uint4*>(kst + r * KROW + c * 16) = val;
     }
     const T* gq = reinterpret_cast<const T*>(lv.guide) + (size_t)unit * nq * D;
@@ -304,8 +356,9 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
         const float inv_nq = 1.f / (float)nq;
         if (!accum) {
             for (int mm = tid; mm < M; mm += blockDim.x) {
+                const int col = all_cols ? mid_slot[mm] : mm;  // (all columns summed: pick the mid entry's slot)
                 float sc = 0.f;
-                for (int w = 0; w < W; ++w) sc += wsum[w * wsum_stride + mm];
+                for (int w = 0; w < W; ++w) sc += wsum[w * wsum_stride + col];
                 sc *= inv_nq;
                 S[mm] = sc;
                 lv.scores[(size_t)unit * lv.mid_pad + mm] = sc;
@@ -317,10 +370,12 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
                 float sc = 0.f;
                 for (int w = 0; w < W; ++w) sc += wsum[w * wsum_stride + sl];
                 sc *= inv_nq;
-                const float total = (sl >= n_stage - n ? 0.f : acc[sl]) + sc;
-                acc[sl] = total;
-                const int mm = sl - mid0;
-                if (compress && mm >= 0 && mm < M) {
+                acc[sl] = (sl >= n_stage - n ? 0.f : acc[sl]) + sc;
+            }
+            __syncthreads();
+            if (compress) {
+                for (int mm = tid; mm < M; mm += blockDim.x) {
+                    const float total = acc[reuse ? mid_slot[mm] : mid0 + mm];
                     S[mm] = total;
                     lv.scores[(size_t)unit * lv.mid_pad + mm] = total;
                 }
@@ -351,6 +406,40 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
     }
     __syncthreads();
 
+    if (reuse) {
+        // ---- Eq. 5-7 without compaction: the n evicted slots take the n rows of the newest line (the last n slots; none
+        // of them is a hole, since the last r >= 1 lines are never evicted), so the cache stays dense
+        if (warp == 0) {
+            int base = 0;
+            for (int m0 = 0; m0 < M; m0 += 32) {
+                const int mm = m0 + lane;
+                const bool ev = mm < M && !keep[mm];
+                const unsigned bal = __ballot_sync(0xffffffffu, ev);
+                if (ev && base + __popc(bal & ((1u << lane) - 1u)) < n) srcmap[base + __popc(bal & ((1u << lane) - 1u))] = mid_slot[mm];
+                base += __popc(bal);
+            }
+        }
+        __syncthreads();
+        const int tail0 = st.len - n;
+        for (int idx = tid; idx < n * CHUNKS; idx += blockDim.x) {
+            const int j = idx / CHUNKS, c = idx - j * CHUNKS;
+            const size_t src = row_offset(lv, unit, tail0 + j, ROW_BYTES) + c * 16, dst = row_offset(lv, unit, srcmap[j], ROW_BYTES) + c * 16;
+            *reinterpret_cast<uint4*>(lv.k_pool + dst) = *reinterpret_cast<const uint4*>(lv.k_pool + src);
+            *reinterpret_cast<uint4*>(lv.v_pool + dst) = *reinterpret_cast<const uint4*>(lv.v_pool + src);
+        }
+        for (int j = tid; j < n; j += blockDim.x) {
+            imap[srcmap[j]] = imap[tail0 + j];
+            if (accum) lv.acc[(size_t)unit * lv.cap_pad + srcmap[j]] = lv.acc[(size_t)unit * lv.cap_pad + tail0 + j];
+        }
+        if (tid == 0) {
+            UnitState ns;
+            ns.len = st.len - n;
+            ns.n_tok = st.n_tok;
+            lv.state[unit] = ns;
+        }
+        return;
+    }
+
     // ---- Eq. 5-6: source slot (relative to mid0) of every row behind the anchor after compaction
     if (warp == 0) {
         int base = 0;
@@ -370,7 +459,6 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
     constexpr int PER_THREAD = 4;
     const int nthr = (int)blockDim.x;
     const int tile_rows = nthr * PER_THREAD / CHUNKS;  // <= nthr
-    int* imap = lv.index_map + (size_t)unit * lv.cap_pad;
     for (int t0 = 0; t0 < total_rows; t0 += tile_rows) {
         const int rows = min(tile_rows, total_rows - t0);
         uint4 kbuf[PER_THREAD], vbuf[PER_THREAD];

@@ -20,6 +20,7 @@ LAR_FLAG_NO_HOST_CHECKS, LAR_FLAG_PDL, LAR_FLAG_SHUFFLE_PAGES, LAR_FLAG_TILE_RAN
 LAR_FLAG_SCORE_CACHE_NORM = 0x10
 LAR_FLAG_HOST_DEFER_OUT = 0x20
 LAR_FLAG_SCORE_ACCUM = 0x40
+LAR_FLAG_SLOT_REUSE = 0x80
 
 
 class lar_config_t(C.Structure):
@@ -69,6 +70,7 @@ def lib():
         "lar_append_kv": (C.c_int, [vp, ip, vp, vp, ip, vp]),
         "lar_decode_attn": (C.c_int, [vp, ip, vp, vp, vp]),
         "lar_decode_step": (C.c_int, [vp, ip, vp, vp, vp, vp, vp]),
+        "lar_decode_step_strided": (C.c_int, [vp, ip, vp, vp, vp, vp, C.c_int64, C.c_int64, C.c_int64, C.c_int64, vp]),
         "lar_decode_step_host": (C.c_int, [vp, ip, vp, vp, vp, vp, vp]),
         "lar_cache_host_join": (C.c_int, [vp, vp]),
         "lar_line_end_score_evict": (C.c_int, [vp, ip, vp]),
@@ -162,6 +164,12 @@ def lar_decode_attn(cache, layer, q, out, stream=None):
 
 def lar_decode_step(cache, layer, q, k, v, out, stream=None):
     _chk(lib().lar_decode_step(cache, layer, _ptr(q), _ptr(k), _ptr(v), _ptr(out), stream), "lar_decode_step")
+
+
+def lar_decode_step_strided(cache, layer, q, k, v, out, q_seq_stride, k_seq_stride, v_seq_stride, out_seq_stride,
+                            stream=None):
+    _chk(lib().lar_decode_step_strided(cache, layer, _ptr(q), _ptr(k), _ptr(v), _ptr(out), q_seq_stride, k_seq_stride,
+                                       v_seq_stride, out_seq_stride, stream), "lar_decode_step_strided")
 
 
 def lar_decode_step_host(cache, layer, q, k, v, out, stream=None):
@@ -266,6 +274,10 @@ class Cache:
 
     def decode_step(self, layer, q, k, v, out):
         lar_decode_step(self.handle, layer, q, k, v, out, self._stream())
+
+    def decode_step_strided(self, layer, q, k, v, out, q_seq_stride, k_seq_stride, v_seq_stride, out_seq_stride):
+        lar_decode_step_strided(self.handle, layer, q, k, v, out, q_seq_stride, k_seq_stride, v_seq_stride,
+                                out_seq_stride, self._stream())
 
     def decode_step_host(self, layer, q, k, v, out):
         lar_decode_step_host(self.handle, layer, q, k, v, out, self._stream())

@@ -69,6 +69,8 @@ def run_parity(w: W.Workload, *, units: Optional[Sequence[Tuple[int, int, int]]]
     dev = torch.device(device)
     cfg = lar.config_from_workload(w, **(cfg_overrides or {}))
     cache = lar.Cache(cfg, device=device)
+    # without compaction the slots do not follow positions: the live SET is what Eq. 5-7 define
+    reuse = bool(cfg.flags & lar.LAR_FLAG_SLOT_REUSE)
     rep = ParityReport(dtype=w.dtype)
     L, S, Hq, Hkv, d, G, n, C = (w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.group,
                                  w.line_width, w.cond_len)
@@ -178,7 +180,10 @@ def run_parity(w: W.Workload, *, units: Optional[Sequence[Tuple[int, int, int]]]
                         else:
                             u.evict(sorted(ev_o))
                     pos_o = u.positions()
-                    if lens[ui] != len(pos_o) or not np.array_equal(imap[ui, : lens[ui]], pos_o):
+                    live = imap[ui, : lens[ui]]
+                    same = (np.array_equal(np.sort(live), pos_o) and len(set(live.tolist())) == len(live)) if reuse \
+                        else np.array_equal(live, pos_o)
+                    if lens[ui] != len(pos_o) or not same:
                         if len(rep.mismatches) < 10:
                             rep.mismatches.append(f"index map layer {l} seq {s} head {h} line {t1 // n}: "
                                                   f"len gpu {lens[ui]} oracle {len(pos_o)}")

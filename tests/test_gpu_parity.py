@@ -255,6 +255,35 @@ def test_cache_normalised_scoring_full_size_sampled(name, layers, n_units, score
     assert rep.compressions == n_units * (w.n_lines - w.budget_lines)
 
 
+# ------------------------------------------------------------------ no compaction: evicted slots are refilled
+@pytest.mark.parametrize("kw", [
+    dict(),                                                             # fp32, G = 1
+    dict(dtype="bf16", head_dim=64, n_q_heads=4, n_kv_heads=2),
+    dict(dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=1, cond_len=0),
+    dict(dtype="bf16", head_dim=64, n_q_heads=4, n_kv_heads=4, cond_len=3, anchor_len=5, recent_lines=2, budget_lines=5),
+    dict(dtype="bf16", head_dim=64, n_q_heads=2, n_kv_heads=2, anchor_len=0, recent_lines=3, budget_lines=6),
+])
+@pytest.mark.parametrize("score_norm", ["mid", "cache", "accum"])
+def test_slot_reuse_keeps_the_same_sets_and_outputs(kw, score_norm):
+    """Under LAR_FLAG_SLOT_REUSE the live set after every line end, every output and every score equal the oracle's;
+    only the order of the slots differs (the harness compares the index map as a set and rejects duplicates)."""
+    w = W.WORKLOADS["tiny_b"].scaled(score_norm=score_norm, **kw)
+    for line_end_all in (False, True):
+        rep = run_parity(w, cfg_overrides=dict(flags=lar.LAR_FLAG_SLOT_REUSE | lar.LAR_FLAG_PDL), line_end_all=line_end_all)
+        _check(rep, w, allow_near_ties=1)
+        assert rep.compressions > 0
+        assert rep.max_score_rel_err < (2e-3 if w.dtype == "bf16" else 1e-4)
+
+
+@pytest.mark.parametrize("name,layers,n_units", [("janus_pro_7b", 2, 4), ("gqa_1024", 1, 3), ("llamagen_xl", 1, 3), ("lumina_768", 1, 3)])
+def test_slot_reuse_full_size_sampled(name, layers, n_units):
+    w = W.WORKLOADS[name].scaled(n_layers=layers)
+    rep = run_parity(w, units=pick_units(w, n_units, seed=4), gen_device="cuda",
+                     cfg_overrides=dict(flags=lar.LAR_FLAG_PDL | lar.LAR_FLAG_SLOT_REUSE), line_end_all=True)
+    _check(rep, w, allow_near_ties=2)
+    assert rep.compressions == n_units * (w.n_lines - w.budget_lines)
+
+
 def test_bf16_mid_region_smaller_than_one_key_tile():
     # M = 6 < 8: some lanes of the scoring warp see no valid key at all in the only tile
     w = W.WORKLOADS["tiny_b"].scaled(dtype="bf16", head_dim=64, n_q_heads=4, n_kv_heads=2, line_width=3, n_lines=12,

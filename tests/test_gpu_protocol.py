@@ -124,6 +124,54 @@ def test_a_key_that_is_not_finite_is_recorded_and_the_line_end_still_evicts_n(dt
     c.close()
 
 
+@pytest.mark.parametrize("n_q_heads,n_kv_heads,head_dim", [(4, 4, 64), (8, 2, 128)])
+def test_strided_views_of_a_fused_qkv_buffer_give_the_same_as_dense_tensors(n_q_heads, n_kv_heads, head_dim):
+    """q, k, v as column ranges of one [batch, (Hq + 2 Hkv) d] buffer and out as a view of a wider buffer: outputs are
+    bit-equal to the dense call's, the caches end in the same state (two line ends, one of them compressing)."""
+    kw = dict(n_layers=1, batch=3, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, head_dim=head_dim, budget_lines=3, n_lines=6)
+    cfg = _small(**kw)
+    ca, cb = lar.Cache(cfg), lar.Cache(cfg)
+    b = _bufs(cfg)
+    for c in (ca, cb):
+        c.append_kv(0, b["kc"], b["vc"], 4)
+    S, d = cfg.batch, head_dim
+    nq, nk = n_q_heads * d, n_kv_heads * d
+    row = nq + 2 * nk
+    g = torch.Generator(device="cpu").manual_seed(3)
+    out_wide = torch.zeros(S, nq + 64, dtype=torch.bfloat16, device="cuda:0")
+    for t in range(4 * 8):
+        qkv = torch.randn(S, row, generator=g).to(torch.bfloat16).to("cuda:0")
+        q, k, v = qkv[:, :nq], qkv[:, nq:nq + nk], qkv[:, nq + nk:]
+        dense_out = torch.zeros(S, n_q_heads, d, dtype=torch.bfloat16, device="cuda:0")
+        ca.decode_step(0, q.contiguous().view(S, n_q_heads, d), k.contiguous().view(S, n_kv_heads, d),
+                       v.contiguous().view(S, n_kv_heads, d), dense_out)
+        out_wide.fill_(float("nan"))
+        cb.decode_step_strided(0, q, k, v, out_wide[:, 32:], row, row, row, nq + 64)
+        torch.cuda.synchronize()
+        assert torch.equal(out_wide[:, 32:32 + nq].reshape(S, n_q_heads, d), dense_out)
+        assert torch.isnan(out_wide[:, :32]).all() and torch.isnan(out_wide[:, 32 + nq:]).all()   # nothing written outside the view
+        if t % 8 == 7:
+            ca.line_end_score_evict(0)
+            cb.line_end_score_evict(0)
+    (la, ia), (lb, ib) = ca.get_state(0), cb.get_state(0)
+    assert (la == lb).all() and (ia == ib).all() and (la == 4 + 3 * 8 - 8).all()   # C + B - n after a compressing line end
+    assert ca.poll_device_status() == 0 and cb.poll_device_status() == 0
+    # strides that are not 16-byte multiples, or shorter than a sequence's heads, are refused
+    assert _status(cb.decode_step_strided, 0, q, k, v, out_wide, row + 4, row, row, nq + 64) == lar.LAR_ERR_INVALID_ARG
+    assert _status(cb.decode_step_strided, 0, q, k, v, out_wide, row, nk - 8, row, nq + 64) == lar.LAR_ERR_INVALID_ARG
+    ca.close()
+    cb.close()
+
+
+def test_strided_entry_point_is_refused_for_fp32_caches():
+    cfg = _small(n_layers=1, dtype="fp32")
+    c = lar.Cache(cfg)
+    b = _bufs(cfg)
+    c.append_kv(0, b["kc"], b["vc"], 4)
+    assert _status(c.decode_step_strided, 0, b["q"], b["k"], b["v"], b["out"], 4 * 64, 4 * 64, 4 * 64, 4 * 64) == lar.LAR_ERR_INVALID_ARG
+    c.close()
+
+
 def test_reset_forgets_deferred_host_copies():
     cfg = _small(n_layers=1, flags=lar.LAR_FLAG_HOST_DEFER_OUT)
     c = lar.Cache(cfg)
