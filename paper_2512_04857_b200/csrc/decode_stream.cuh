@@ -239,21 +239,22 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     // dependent's wait covers this whole grid (which itself waits for its predecessor below).
     grid_dep_launch();
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < NS; ++s) {
-            mbar_init(bar_full + s * 8, 1);
-            mbar_init(bar_empty + s * 8, 1);
+    {
+        // one barrier per thread (the set-up of a launch is on the path between two launches)
+        const int t = (int)threadIdx.x;
+        if (t < 2 * NS) {
+            mbar_init(bar_full + t * 8, 1);  // full / empty of the K/V ring (adjacent in memory)
+        } else if (t < 2 * NS + NQ) {
+            mbar_init(bar_qfull + (t - 2 * NS) * 8, 1);
+        } else if (t < 2 * NS + 2 * NQ) {
+            mbar_init(bar_qempty + (t - 2 * NS - NQ) * 8, (uint32_t)(W + 1));
+        } else if (t < 2 * NS + 2 * NQ + 2) {
+            mbar_init(bar_pfull + (t - 2 * NS - 2 * NQ) * 8, (uint32_t)W);
+        } else if (t < 2 * NS + 2 * NQ + 4) {
+            mbar_init(bar_pempty + (t - 2 * NS - 2 * NQ - 2) * 8, 1);
         }
-        for (int s = 0; s < NQ; ++s) {
-            mbar_init(bar_qfull + s * 8, 1);
-            mbar_init(bar_qempty + s * 8, (uint32_t)(W + 1));
-        }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(bar_pfull + s * 8, (uint32_t)W);
-            mbar_init(bar_pempty + s * 8, 1);
-        }
-        *abort_flag = 0;
-        mbar_fence_init();
+        if (t == 0) *abort_flag = 0;
+        if (t < 2 * NS + 2 * NQ + 4) mbar_fence_init();
     }
     __syncthreads();
 
@@ -564,6 +565,18 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         if (!ok && lane == 0) atomicOr(lv.status, kStWaitLimit);
     } else {
         // =========================================================================== epilogue
+        if (a.prefetch) {
+            // a hint only (L2 is the point of coherence): the step's inputs start their way from HBM before the dependency
+            // resolves, if the kernel that produced them has not left them in L2 anyway
+            for (int sg = lane; sg < n_segs; sg += 32) {
+                const int un = u0 + sg;
+                l2_prefetch_bulk(reinterpret_cast<const T16*>(a.q) + unit_offset(un, a.q_seq_stride, G * D), G * D * 2);
+                if (a.fused && (un + 1) * T <= t_end) {
+                    l2_prefetch_bulk(reinterpret_cast<const T16*>(a.k_new) + unit_offset(un, a.k_seq_stride, D), D * 2);
+                    l2_prefetch_bulk(reinterpret_cast<const T16*>(a.v_new) + unit_offset(un, a.v_seq_stride, D), D * 2);
+                }
+            }
+        }
         grid_dep_wait();
         if (p == 0 && lane == 0) st_release_gpu(a.done_seq, a.seq - 1);  // everything before this launch has completed
         bool ok = true;
