@@ -145,7 +145,13 @@ constexpr int kMaxConsumers = 6;  // consumer warps per CTA at most
 constexpr int kProducers = 2;     // producer warps per CTA: tile j is fetched by producer j % kProducers
 constexpr int kMaxQSlots = 8;     // depth of the query ring at most
 // query ring / partial buffers of a CTA that works on at most `segs` segments per launch
-__host__ __device__ constexpr int stream_q_slots(int G, int segs) { const int q = G <= 2 ? 8 : 4; return segs < q ? (segs < 1 ? 1 : segs) : q; }
+// (a power of two, so that ring positions are masks and shifts: every warp takes them once per segment)
+__host__ __device__ constexpr int stream_q_slots(int G, int segs) {
+    const int q = G <= 2 ? 8 : 4;
+    int r = 1;
+    while (2 * r <= segs && 2 * r <= q) r *= 2;
+    return r;
+}
 __host__ __device__ constexpr int stream_partial_bufs(int segs) { return segs < 2 ? 1 : 2; }
 __host__ __device__ constexpr int stream_q_entry_bytes(int D, int G) { return ((G + 2) * D * 2 + 127) / 128 * 128; }
 __host__ __device__ constexpr int stream_fixed_smem_bytes(int D, int G, int W, int NQ, int NPB) {
@@ -210,7 +216,8 @@ template <int D, int G>
 __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs a, const __grid_constant__ TensorMaps tm) {
     using TR = MmaTraits<D>;
     using T16 = __nv_bfloat16;
-    const int NQ = a.q_slots, NPB = a.p_bufs;
+    const int NQ = a.q_slots, NPB = a.p_bufs;  // powers of two
+    const int qsh = __ffs(NQ) - 1, psh = NPB - 1;
     constexpr int QENT = stream_q_entry_bytes(D, G);
     constexpr int PS = D + 2;  // floats per (warp, head) partial: o[D], m, l
     constexpr int PER = D / 32;
@@ -292,8 +299,8 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         return (size_t)sq * (size_t)seq_stride + (size_t)(u - sq * lv.n_kv_heads) * per_head;
     };
     auto issue_inputs = [&](int seg) -> bool {
-        const int slot = seg % NQ;
-        if (seg >= NQ && !wait_or_abort(bar_qempty + slot * 8, (uint32_t)((seg / NQ - 1) & 1), abort_flag)) return false;
+        const int slot = seg & (NQ - 1);
+        if (seg >= NQ && !wait_or_abort(bar_qempty + slot * 8, (uint32_t)(((seg >> qsh) - 1) & 1), abort_flag)) return false;
         const int unit = u0 + seg;
         const bool closes = (unit + 1) * T <= t_end;  // the segment holds the unit's last tile
         const bool with_kv = a.fused && closes;
@@ -407,8 +414,8 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             const int je = (ub + T < t_end ? ub + T : t_end) - t_begin;
 
             // ---- Q fragments (A operand): row qrow = head, 16 columns per k-step; heads >= G are zero rows
-            const int qs = seg % NQ;
-            ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag);
+            const int qs = seg & (NQ - 1);
+            ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)(((seg >> qsh)) & 1), abort_flag);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             uint32_t qa0[TR::KSTEPS], qa2[TR::KSTEPS];
             {
@@ -524,9 +531,9 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             if (!ok) break;
 
             // ---- this warp's partial of the segment -> shared memory
-            const int buf = seg % NPB;
+            const int buf = seg & (NPB - 1);
             if (seg >= NPB) {
-                ok = wait_or_abort(bar_pempty + buf * 8, (uint32_t)((seg / NPB - 1) & 1), abort_flag);
+                ok = wait_or_abort(bar_pempty + buf * 8, (uint32_t)(((seg >> psh) - 1) & 1), abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             }
 #pragma unroll
@@ -566,9 +573,10 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     } else {
         // =========================================================================== epilogue
         if (a.prefetch) {
-            // a hint only (L2 is the point of coherence): the step's inputs start their way from HBM before the dependency
-            // resolves, if the kernel that produced them has not left them in L2 anyway
-            for (int sg = lane; sg < n_segs; sg += 32) {
+            // a hint only (L2 is the point of coherence): the inputs of the first segments -- the ones the launch waits for
+            // -- start their way from HBM before the dependency resolves, if the kernel that produced them has not left
+            // them in L2 anyway
+            for (int sg = lane; sg < n_segs && sg < NQ; sg += 32) {
                 const int un = u0 + sg;
                 l2_prefetch_bulk(reinterpret_cast<const T16*>(a.q) + unit_offset(un, a.q_seq_stride, G * D), G * D * 2);
                 if (a.fused && (un + 1) * T <= t_end) {
@@ -606,9 +614,9 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             const int ub = unit * T;
             const bool opens = ub >= t_begin, closes = ub + T <= t_end;
             const size_t out_base = unit_offset(unit, a.out_seq_stride, G * D);
-            const int qs = seg % NQ, buf = seg % NPB;
+            const int qs = seg & (NQ - 1), buf = seg & (NPB - 1);
             closing_loads(seg + 1, page_nxt, dev_len_nxt);
-            ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)((seg / NQ) & 1), abort_flag);
+            ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)(((seg >> qsh)) & 1), abort_flag);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             const unsigned char* Qs = qring_ptr + qs * QENT;
             const uint16_t* Q16 = reinterpret_cast<const uint16_t*>(Qs);
@@ -680,7 +688,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             if (lane == 0) mbar_arrive(bar_qempty + qs * 8);
 
             // ---- merge the consumers' partials (+ the step's token)
-            ok = wait_or_abort(bar_pfull + buf * 8, (uint32_t)((seg / NPB) & 1), abort_flag);
+            ok = wait_or_abort(bar_pfull + buf * 8, (uint32_t)(((seg >> psh)) & 1), abort_flag);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             const float* pb = pbuf + buf * pbuf_floats;
             // branch-free and unrolled over the (at most kMaxConsumers) consumer warps, so that the shared-memory
