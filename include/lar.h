@@ -194,6 +194,19 @@ lar_status_t lar_decode_step_strided(lar_cache_t* c, int layer, const void* q, c
                                      int64_t q_seq_stride, int64_t k_seq_stride, int64_t v_seq_stride,
                                      int64_t out_seq_stride, void* stream);
 
+/* lar_decode_step_strided with the rotary position embedding of q and k fused in (bf16 storage only): the kernel rotates
+ * the G query rows of every unit and the new key row before anything else uses them, so the cache receives rotated keys
+ * and the guide queue rotated queries -- the space in which Eq. 8-9 compare them (Sec. 3.3) -- without a separate pass
+ * over q and k.  cos_sin: device, fp32, [batch, head_dim]: for each sequence the cosines of the head_dim / 2 rotation
+ * angles of this step's position, then the sines.  interleaved = 0 rotates the pairs (i, i + head_dim / 2), interleaved
+ * != 0 the pairs (2 i, 2 i + 1):
+ *     x' = x cos_i - y sin_i,  y' = y cos_i + x sin_i     (fp32, every product and sum rounded, result rounded to bf16)
+ * v is not rotated.  Strides, alignment, call order and errors as lar_decode_step_strided (pass the dense row lengths
+ * for dense tensors). */
+lar_status_t lar_decode_step_rope(lar_cache_t* c, int layer, const void* q, const void* k, const void* v, void* out,
+                                  int64_t q_seq_stride, int64_t k_seq_stride, int64_t v_seq_stride, int64_t out_seq_stride,
+                                  const float* cos_sin, int interleaved, void* stream);
+
 /* lar_decode_step with HOST buffers (pinned memory): copies q, k, v to a staging area of the slab, runs the
  * fused kernel and copies `out` back, asynchronously.  Seen from `stream` the call is one stream-ordered
  * operation: `out_host` is complete once work enqueued on `stream` after the call runs (or `stream` is

@@ -59,6 +59,8 @@ struct StreamArgs {
     float scale_log2;   // softmax scale * log2(e)
     int len, n_tok;     // live rows per unit / visual tokens appended so far, before this step's append
     int unit_ranges;    // 1: CTA ranges end on unit boundaries
+    const float* rope;  // rotary embedding: [sequence][d] floats, cos of the d/2 pairs then sin, for this step's position
+    int rope_mode;      // 0: none; 1: pairs (i, i + d/2); 2: pairs (2 i, 2 i + 1)
     int fused;          // 1: the step's token comes from k_new / v_new and is appended by this kernel
     int prefetch;       // 1: the CTA may fill its ring before waiting for the preceding kernel (units whose length is published)
     int n_units, n_stages, max_seg;
@@ -158,7 +160,7 @@ __host__ __device__ constexpr int stream_fixed_smem_bytes(int D, int G, int W, i
     return 1024                                  // slack: the ring starts on a 1024-byte boundary
            + NQ * stream_q_entry_bytes(D, G)     // query ring
            + NPB * (W + 1) * G * (D + 2) * 4     // partial buffers
-           + (2 * kMaxQSlots + 4) * 8 + 16;      // query / partial barriers, abort flag
+           + (3 * kMaxQSlots + 4) * 8 + 16;      // query / partial barriers, abort flag
 }
 __host__ __device__ constexpr int stream_smem_bytes(int D, int G, int W, int NS, int NQ, int NPB) {
     return stream_fixed_smem_bytes(D, G, W, NQ, NPB) + NS * (2 * (D / 64) * kStreamTile * 128 + 16);  // stage + its 2 barriers
@@ -240,7 +242,10 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     const uint32_t bar_full = bars, bar_empty = bars + NS * 8;
     const uint32_t bar_qfull = bars + 2 * NS * 8, bar_qempty = bar_qfull + kMaxQSlots * 8;
     const uint32_t bar_pfull = bar_qempty + kMaxQSlots * 8, bar_pempty = bar_pfull + 2 * 8;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_ptr + (2 * NS + 2 * kMaxQSlots + 4) * 8);
+    const uint32_t bar_qrot = bar_pempty + 2 * 8;  // (rotary embedding) the slot's q and k rows have been rotated
+    // what the consumers wait for before they take a segment's queries
+    const uint32_t bar_qready = a.rope_mode ? bar_qrot : bar_qfull;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_ptr + (2 * NS + 3 * kMaxQSlots + 4) * 8);
 
     // Dependents may be scheduled from now on: they only hint the L2 before their own griddepcontrol.wait, and a
     // dependent's wait covers this whole grid (which itself waits for its predecessor below).
@@ -259,9 +264,11 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             mbar_init(bar_pfull + (t - 2 * NS - 2 * NQ) * 8, (uint32_t)W);
         } else if (t < 2 * NS + 2 * NQ + 4) {
             mbar_init(bar_pempty + (t - 2 * NS - 2 * NQ - 2) * 8, 1);
+        } else if (t < 2 * NS + 3 * NQ + 4) {
+            mbar_init(bar_qrot + (t - 2 * NS - 2 * NQ - 4) * 8, 1);
         }
         if (t == 0) *abort_flag = 0;
-        if (t < 2 * NS + 2 * NQ + 4) mbar_fence_init();
+        if (t < 2 * NS + 3 * NQ + 4) mbar_fence_init();
     }
     __syncthreads();
 
@@ -415,7 +422,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
 
             // ---- Q fragments (A operand): row qrow = head, 16 columns per k-step; heads >= G are zero rows
             const int qs = seg & (NQ - 1);
-            ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)(((seg >> qsh)) & 1), abort_flag);
+            ok = wait_or_abort(bar_qready + qs * 8, (uint32_t)(((seg >> qsh)) & 1), abort_flag);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             uint32_t qa0[TR::KSTEPS], qa2[TR::KSTEPS];
             {
@@ -616,10 +623,40 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             const size_t out_base = unit_offset(unit, a.out_seq_stride, G * D);
             const int qs = seg & (NQ - 1), buf = seg & (NPB - 1);
             closing_loads(seg + 1, page_nxt, dev_len_nxt);
+            // rotary embedding: cos and sin of this sequence's position for the pairs this lane rotates (on their way
+            // while the inputs arrive)
+            float rc[D / 64], rs[D / 64];
+            if (a.rope_mode) {
+                const float* cs = a.rope + (size_t)(unit / lv.n_kv_heads) * D;
+#pragma unroll
+                for (int k = 0; k < D / 64; ++k) {
+                    rc[k] = __ldg(cs + lane + 32 * k);
+                    rs[k] = __ldg(cs + D / 2 + lane + 32 * k);
+                }
+            }
             ok = wait_or_abort(bar_qfull + qs * 8, (uint32_t)(((seg >> qsh)) & 1), abort_flag);
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             const unsigned char* Qs = qring_ptr + qs * QENT;
             const uint16_t* Q16 = reinterpret_cast<const uint16_t*>(Qs);
+            if (a.rope_mode) {
+                // q (all G heads) and the new k row are rotated in place, pair by pair, in fp32 with every product and
+                // sum rounded separately, then rounded to bf16: the cache, the guide queue and the logits see rotated rows
+                T16* rows = reinterpret_cast<T16*>(qring_ptr + qs * QENT);
+                const int n_rows = G + ((a.fused && closes) ? 1 : 0);
+                for (int r = 0; r < n_rows; ++r) {
+#pragma unroll
+                    for (int k = 0; k < D / 64; ++k) {
+                        const int i = lane + 32 * k;  // pair: (i, i + d/2), or (2 i, 2 i + 1) in the interleaved convention
+                        const int ia = a.rope_mode == 1 ? i : 2 * i, ib = a.rope_mode == 1 ? i + D / 2 : 2 * i + 1;
+                        const float x = __bfloat162float(rows[r * D + ia]), y = __bfloat162float(rows[r * D + ib]);
+                        rows[r * D + ia] = __float2bfloat16_rn(__fsub_rn(__fmul_rn(x, rc[k]), __fmul_rn(y, rs[k])));
+                        rows[r * D + ib] = __float2bfloat16_rn(__fadd_rn(__fmul_rn(y, rc[k]), __fmul_rn(x, rs[k])));
+                    }
+                }
+                fence_proxy_async_smem();  // these writes come before the copy that refills the slot
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_qrot + qs * 8);
+            }
 
             // ---- the token of this step (Eq. 4, 8): logit per head, value row, stores
             // Merge layout: the warp's lanes are split over the G heads, LPH lanes per head; lane (hg, sub) owns the

@@ -456,6 +456,8 @@ lar_status_t launch_append(lar_cache* c, int layer, const void* k, const void* v
 // Elements between consecutive sequences of q, k, v and out (0 = dense).
 struct SeqStrides {
     long long q = 0, k = 0, v = 0, out = 0;
+    const float* rope = nullptr;  // rotary embedding applied to q and k by the kernel (nullptr: none)
+    int rope_mode = 0;
 };
 
 lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k, const void* v, void* out, int fused,
@@ -521,6 +523,8 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
         a.k_seq_stride = ss.k;
         a.v_seq_stride = ss.v;
         a.out_seq_stride = ss.out;
+        a.rope = ss.rope;
+        a.rope_mode = ss.rope_mode;
         lc.gridDim = dim3((unsigned)c->d.ctas, 1, 1);
         lc.blockDim = dim3((unsigned)(32 * (c->plan.warps_per_cta + lar::kProducers + 1)), 1, 1);
         lc.attrs = attrs;
@@ -528,7 +532,7 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
         DecodeStreamFn fn = decode_stream_fn(c->cfg, c->d.group);
         LAR_CUDA(cudaLaunchKernelEx(&lc, fn, a, c->tmaps));
     } else {
-        if (ss.q || ss.k || ss.v || ss.out) return LAR_ERR_INVALID_ARG;  // fp32 storage: dense tensors only
+        if (ss.q || ss.k || ss.v || ss.out || ss.rope) return LAR_ERR_INVALID_ARG;  // fp32 storage: dense tensors only
         lar::DecodeArgs a;
         a.lv = view_of(c, layer);
         a.q = q;
@@ -770,9 +774,27 @@ lar_status_t lar_decode_step(lar_cache_t* c, int layer, const void* q, const voi
     return LAR_OK;
 }
 
+static lar_status_t decode_step_views(lar_cache_t* c, int layer, const void* q, const void* k, const void* v, void* out,
+                                      int64_t q_seq_stride, int64_t k_seq_stride, int64_t v_seq_stride, int64_t out_seq_stride,
+                                      const float* rope, int rope_mode, void* stream);
+
 lar_status_t lar_decode_step_strided(lar_cache_t* c, int layer, const void* q, const void* k, const void* v, void* out,
                                      int64_t q_seq_stride, int64_t k_seq_stride, int64_t v_seq_stride, int64_t out_seq_stride,
                                      void* stream) {
+    return decode_step_views(c, layer, q, k, v, out, q_seq_stride, k_seq_stride, v_seq_stride, out_seq_stride, nullptr, 0, stream);
+}
+
+lar_status_t lar_decode_step_rope(lar_cache_t* c, int layer, const void* q, const void* k, const void* v, void* out,
+                                  int64_t q_seq_stride, int64_t k_seq_stride, int64_t v_seq_stride, int64_t out_seq_stride,
+                                  const float* cos_sin, int interleaved, void* stream) {
+    if (!cos_sin || (reinterpret_cast<uintptr_t>(cos_sin) & 3u)) return LAR_ERR_INVALID_ARG;
+    return decode_step_views(c, layer, q, k, v, out, q_seq_stride, k_seq_stride, v_seq_stride, out_seq_stride, cos_sin,
+                             interleaved ? 2 : 1, stream);
+}
+
+static lar_status_t decode_step_views(lar_cache_t* c, int layer, const void* q, const void* k, const void* v, void* out,
+                                      int64_t q_seq_stride, int64_t k_seq_stride, int64_t v_seq_stride, int64_t out_seq_stride,
+                                      const float* rope, int rope_mode, void* stream) {
     if (bad_layer(c, layer) || !q || !k || !v || !out) return LAR_ERR_INVALID_ARG;
     if (c->cfg.dtype != LAR_BF16) return LAR_ERR_INVALID_ARG;
     const int64_t d = c->cfg.head_dim, hq = c->cfg.n_q_heads, hkv = c->cfg.n_kv_heads;
@@ -788,6 +810,8 @@ lar_status_t lar_decode_step_strided(lar_cache_t* c, int layer, const void* q, c
     ss.k = k_seq_stride == hkv * d ? 0 : k_seq_stride;
     ss.v = v_seq_stride == hkv * d ? 0 : v_seq_stride;
     ss.out = out_seq_stride == hq * d ? 0 : out_seq_stride;
+    ss.rope = rope;
+    ss.rope_mode = rope_mode;
     st = launch_decode(c, layer, q, k, v, out, 1, (cudaStream_t)stream, ss);
     if (st != LAR_OK) return st;
     sh.v += 1;

@@ -71,6 +71,7 @@ def lib():
         "lar_decode_attn": (C.c_int, [vp, ip, vp, vp, vp]),
         "lar_decode_step": (C.c_int, [vp, ip, vp, vp, vp, vp, vp]),
         "lar_decode_step_strided": (C.c_int, [vp, ip, vp, vp, vp, vp, C.c_int64, C.c_int64, C.c_int64, C.c_int64, vp]),
+        "lar_decode_step_rope": (C.c_int, [vp, ip, vp, vp, vp, vp, C.c_int64, C.c_int64, C.c_int64, C.c_int64, vp, ip, vp]),
         "lar_decode_step_host": (C.c_int, [vp, ip, vp, vp, vp, vp, vp]),
         "lar_cache_host_join": (C.c_int, [vp, vp]),
         "lar_line_end_score_evict": (C.c_int, [vp, ip, vp]),
@@ -170,6 +171,13 @@ def lar_decode_step_strided(cache, layer, q, k, v, out, q_seq_stride, k_seq_stri
                             stream=None):
     _chk(lib().lar_decode_step_strided(cache, layer, _ptr(q), _ptr(k), _ptr(v), _ptr(out), q_seq_stride, k_seq_stride,
                                        v_seq_stride, out_seq_stride, stream), "lar_decode_step_strided")
+
+
+def lar_decode_step_rope(cache, layer, q, k, v, out, q_seq_stride, k_seq_stride, v_seq_stride, out_seq_stride, cos_sin,
+                         interleaved, stream=None):
+    _chk(lib().lar_decode_step_rope(cache, layer, _ptr(q), _ptr(k), _ptr(v), _ptr(out), q_seq_stride, k_seq_stride,
+                                    v_seq_stride, out_seq_stride, _ptr(cos_sin), int(interleaved), stream),
+         "lar_decode_step_rope")
 
 
 def lar_decode_step_host(cache, layer, q, k, v, out, stream=None):
@@ -278,6 +286,11 @@ class Cache:
     def decode_step_strided(self, layer, q, k, v, out, q_seq_stride, k_seq_stride, v_seq_stride, out_seq_stride):
         lar_decode_step_strided(self.handle, layer, q, k, v, out, q_seq_stride, k_seq_stride, v_seq_stride,
                                 out_seq_stride, self._stream())
+
+    def decode_step_rope(self, layer, q, k, v, out, q_seq_stride, k_seq_stride, v_seq_stride, out_seq_stride, cos_sin,
+                         interleaved=False):
+        lar_decode_step_rope(self.handle, layer, q, k, v, out, q_seq_stride, k_seq_stride, v_seq_stride, out_seq_stride,
+                             cos_sin, interleaved, self._stream())
 
     def decode_step_host(self, layer, q, k, v, out):
         lar_decode_step_host(self.handle, layer, q, k, v, out, self._stream())

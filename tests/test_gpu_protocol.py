@@ -163,6 +163,60 @@ def test_strided_views_of_a_fused_qkv_buffer_give_the_same_as_dense_tensors(n_q_
     cb.close()
 
 
+def _rotate(x, cos, sin, interleaved):
+    """Rotary embedding of x [S, H, d] (bf16) with cos, sin [S, d/2] (fp32), rounded like the kernel: fp32 products and
+    sums, each rounded, result to bf16."""
+    S, H, d = x.shape
+    xf = x.float()
+    a, b = (xf[..., 0::2], xf[..., 1::2]) if interleaved else (xf[..., : d // 2], xf[..., d // 2:])
+    c, s_ = cos[:, None, :], sin[:, None, :]
+    ra, rb = a * c - b * s_, b * c + a * s_
+    out = torch.empty_like(xf)
+    if interleaved:
+        out[..., 0::2], out[..., 1::2] = ra, rb
+    else:
+        out[..., : d // 2], out[..., d // 2:] = ra, rb
+    return out.to(torch.bfloat16)
+
+
+@pytest.mark.parametrize("n_q_heads,n_kv_heads,head_dim,interleaved", [(4, 4, 64, False), (8, 2, 128, False), (4, 2, 128, True)])
+def test_fused_rotary_embedding_equals_rotating_first(n_q_heads, n_kv_heads, head_dim, interleaved):
+    """lar_decode_step_rope on raw q, k against lar_decode_step on q, k rotated beforehand with the same arithmetic:
+    outputs bit-equal, the caches evict the same tokens (the guide queue and the cached keys hold rotated rows)."""
+    kw = dict(n_layers=1, batch=3, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, head_dim=head_dim, budget_lines=3, n_lines=6)
+    cfg = _small(**kw)
+    ca, cb = lar.Cache(cfg), lar.Cache(cfg)
+    b = _bufs(cfg)
+    for c in (ca, cb):
+        c.append_kv(0, b["kc"], b["vc"], 4)
+    S, d = cfg.batch, head_dim
+    g = torch.Generator(device="cpu").manual_seed(11)
+    mk = lambda *s: torch.randn(*s, generator=g).to(torch.bfloat16).to("cuda:0")
+    inv_freq = 1.0 / (10000.0 ** (torch.arange(d // 2, dtype=torch.float32) / (d // 2)))
+    for t in range(5 * 8):
+        q, k, v = mk(S, n_q_heads, d), mk(S, n_kv_heads, d), mk(S, n_kv_heads, d)
+        pos = torch.tensor([t + 3 * s_ for s_ in range(S)], dtype=torch.float32)      # a position per sequence
+        ang = pos[:, None] * inv_freq[None, :]
+        cos, sin = torch.cos(ang).to("cuda:0"), torch.sin(ang).to("cuda:0")
+        cos_sin = torch.cat([cos, sin], dim=1).contiguous()
+        oa = torch.zeros(S, n_q_heads, d, dtype=torch.bfloat16, device="cuda:0")
+        ob = torch.zeros_like(oa)
+        ca.decode_step(0, _rotate(q, cos, sin, interleaved), _rotate(k, cos, sin, interleaved), v, oa)
+        cb.decode_step_rope(0, q, k, v, ob, n_q_heads * d, n_kv_heads * d, n_kv_heads * d, n_q_heads * d, cos_sin, interleaved)
+        torch.cuda.synchronize()
+        assert torch.equal(oa, ob), f"step {t}: max diff {(oa.float() - ob.float()).abs().max().item()}"
+        if t % 8 == 7:
+            ca.line_end_score_evict(0)
+            cb.line_end_score_evict(0)
+    (la, ia), (lb, ib) = ca.get_state(0), cb.get_state(0)
+    assert (la == lb).all() and (ia == ib).all()
+    assert ca.poll_device_status() == 0 and cb.poll_device_status() == 0
+    assert _status(cb.decode_step_rope, 0, q, k, v, ob, n_q_heads * d, n_kv_heads * d, n_kv_heads * d, n_q_heads * d, None,
+                   interleaved) == lar.LAR_ERR_INVALID_ARG
+    ca.close()
+    cb.close()
+
+
 def test_strided_entry_point_is_refused_for_fp32_caches():
     cfg = _small(n_layers=1, dtype="fp32")
     c = lar.Cache(cfg)
