@@ -60,6 +60,7 @@ struct Derived {
     int unit_ranges;    // bf16 decode: 1 if the CTAs' ranges end on unit boundaries
     int q_slots, p_bufs;  // bf16 decode: depth of a CTA's query ring, number of its partial buffers
     int le_threads;     // threads per CTA of the line-end kernel
+    int le_guide_global;  // line-end kernel: the guide rows are read from global memory instead of being staged
 };
 
 constexpr int kDefaultDecodeCtas = 148;  // one per SM of a B200
@@ -144,6 +145,7 @@ bool derive(const lar_config_t* c, Derived& d) {
     // A unit of T tiles is cut into at most ceil(T / floor(U T / P)) + 1 segments (never more than T or P).
     // line end: one CTA per unit, 8 warps; few units with a large mid region get one warp per 16 guide rows (16..32 warps)
     d.le_threads = 256;
+    d.le_guide_global = 0;
     // (a column sum per warp over every live row -- accumulated attention, or the cache-normalised form without
     // compaction -- stays at 8 warps so that it fits into shared memory)
     const bool all_cols = (c->flags & LAR_FLAG_SCORE_ACCUM) ||
@@ -258,12 +260,21 @@ lar_status_t plan_query_impl(const lar_config_t* cfg, lar_plan_t* out, Derived* 
     p.mid_len = d.M;
     p.compressing = d.compressing;
     choose_plan(cfg, d, p);
-    p.line_end_smem_bytes =
-        d.compressing ? lar::line_end_smem_bytes(d.row_bytes, cfg->head_dim, d.M, d.M - cfg->line_width + cfg->recent_lines * cfg->line_width, d.le_threads / 32,
-                                                 cfg->line_width * d.group, cfg->dtype == LAR_BF16 ? 1 : 0, cfg->cond_len + d.B,
-                                                 (cfg->flags & (LAR_FLAG_SCORE_CACHE_NORM | LAR_FLAG_SCORE_ACCUM)) ? 1 : 0,
-                                                 (cfg->flags & LAR_FLAG_SCORE_ACCUM) ? 1 : 0,
-                                                 (cfg->flags & LAR_FLAG_SLOT_REUSE) ? 1 : 0, d.N) : 0;
+    auto le_bytes = [&]() {
+        return lar::line_end_smem_bytes(d.row_bytes, cfg->head_dim, d.M, d.M - cfg->line_width + cfg->recent_lines * cfg->line_width, d.le_threads / 32,
+                                        cfg->line_width * d.group, cfg->dtype == LAR_BF16 ? 1 : 0, cfg->cond_len + d.B,
+                                        (cfg->flags & (LAR_FLAG_SCORE_CACHE_NORM | LAR_FLAG_SCORE_ACCUM)) ? 1 : 0,
+                                        (cfg->flags & LAR_FLAG_SCORE_ACCUM) ? 1 : 0, (cfg->flags & LAR_FLAG_SLOT_REUSE) ? 1 : 0, d.N,
+                                        d.le_guide_global);
+    };
+    p.line_end_smem_bytes = d.compressing ? le_bytes() : 0;
+    if (p.line_end_smem_bytes > 227 * 1024 && cfg->dtype == LAR_BF16 &&
+        !(cfg->flags & (LAR_FLAG_SCORE_CACHE_NORM | LAR_FLAG_SCORE_ACCUM))) {
+        // a mid region too large to stage next to the guide rows: 8 warps, guide rows read from global memory
+        d.le_threads = 256;
+        d.le_guide_global = 1;
+        p.line_end_smem_bytes = le_bytes();
+    }
     p.slab_bytes = L.total;
     p.scratch_bytes = (L.off_tickets + L.tickets_bytes) - L.off_partials;
     if (p.decode_smem_bytes > 227 * 1024 || p.line_end_smem_bytes > 227 * 1024) return LAR_ERR_INVALID_ARG;
@@ -918,7 +929,7 @@ lar_status_t lar_cache_host_join(lar_cache_t* c, void* stream) {
 // scoring mode of the line-end kernel: bit 0 softmax over the whole live cache, bit 1 accumulated attention
 static int line_end_mode(const lar_cache* c) {
     return ((c->cfg.flags & LAR_FLAG_SCORE_CACHE_NORM) ? 1 : 0) | ((c->cfg.flags & LAR_FLAG_SCORE_ACCUM) ? 2 : 0) |
-           ((c->cfg.flags & LAR_FLAG_SLOT_REUSE) ? 4 : 0);
+           ((c->cfg.flags & LAR_FLAG_SLOT_REUSE) ? 4 : 0) | (c->d.le_guide_global ? 8 : 0);
 }
 
 static lar::LayerStrides layer_strides(const lar_cache* c) {

@@ -55,11 +55,12 @@ __host__ __device__ inline int line_end_staged_rows(int M, int live_rows, int ca
 // reuse (the evicted slots are refilled, nothing is compacted): the mid entries are found through the index map; their
 // slots and a bitmap of the mid positions (n_visual bits, with word-wise prefix counts) are kept in shared memory as well.
 __host__ __device__ inline int line_end_smem_bytes(int row_bytes, int D, int M, int total_rows, int warps, int nq, int is_bf16,
-                                                   int live_rows, int cache_norm, int accum, int reuse, int n_visual) {
+                                                   int live_rows, int cache_norm, int accum, int reuse, int n_visual,
+                                                   int guide_global = 0) {
     const int cols = (accum || (reuse && cache_norm)) ? live_rows : M;  // columns whose probabilities are summed
     int b = line_end_staged_rows(M, live_rows, cache_norm) * (row_bytes + 16);  // keys, rows padded by one chunk against bank conflicts
     if (is_bf16)
-        b += (cache_norm ? 0 : ((nq + 15) / 16 * 16) * (row_bytes + 16)) + warps * cols * 4;  // guide rows (whole 16-row tiles), column sums per warp
+        b += ((cache_norm || guide_global) ? 0 : ((nq + 15) / 16 * 16) * (row_bytes + 16)) + warps * cols * 4;  // guide rows (whole 16-row tiles), column sums per warp
     else
         b += warps * (D + (cache_norm ? live_rows : M) + cols) * 4;  // per warp: query row (fp32), logits row, score accumulator
     b += M * 4;                            // final scores
@@ -78,7 +79,7 @@ __host__ __device__ inline int line_end_smem_bytes(int row_bytes, int D, int M, 
 //   CACHE = true:  keys holds all n_keys live rows, the mid ones from row mid_off; guide row (t, g) is normalised over
 //                  the keys that were live when token t of the line was decoded (rows < n_keys - n + t + 1) and read
 //                  from global memory (gq32: rows of D / 2 words).
-template <int D, bool CACHE>
+template <int D, bool CACHE, bool GQ_GLOBAL = CACHE>
 __device__ __forceinline__ void score_mma(const unsigned char* keys, const unsigned char* qg, const uint32_t* gq32, float* colsum,
                                           int n_keys, int mid_off, int M, int nq, int G, int n, float scale_log2, int warp,
                                           int lane, int W) {
@@ -91,7 +92,7 @@ __device__ __forceinline__ void score_mma(const unsigned char* keys, const unsig
         uint32_t a[KSTEPS][4];
 #pragma unroll
         for (int ks = 0; ks < KSTEPS; ++ks) {
-            if constexpr (CACHE) {
+            if constexpr (GQ_GLOBAL) {
                 a[ks][0] = r0 < nq ? __ldg(gq32 + (size_t)r0 * (D / 2) + ks * 8 + quad) : 0u;
                 a[ks][1] = r1 < nq ? __ldg(gq32 + (size_t)r1 * (D / 2) + ks * 8 + quad) : 0u;
                 a[ks][2] = r0 < nq ? __ldg(gq32 + (size_t)r0 * (D / 2) + ks * 8 + 4 + quad) : 0u;
@@ -200,7 +201,8 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
     // steps (the per-line sums of the cache-normalised form, added up line by line in lv.acc)
     // bit 2: no compaction -- the n evicted slots take the n rows of the newest line (n rows move instead of every row
     // behind the first hole); slots then no longer follow positions, and the mid region is found through the index map
-    const bool accum = (mode & 2) != 0, reuse = (mode & 4) != 0;
+    // bit 3: the guide rows are not staged in shared memory (a mid region too large to stage both): read from global
+    const bool accum = (mode & 2) != 0, reuse = (mode & 4) != 0, guide_global = (mode & 8) != 0;
     const int cache_norm = (mode & 1) | (accum ? 1 : 0);
     const bool compress = v == B;
     if (!compress && !accum) return;  // cache below budget: nothing to evict (the queue restarts by itself)
@@ -224,7 +226,7 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
     // columns whose probabilities are summed: the M mid keys, or (accum) every staged row
     const bool all_cols = accum || (reuse && cache_norm);
     const int cols = all_cols ? n_stage : M, col_off = all_cols ? 0 : mid_off;
-    float* colsum = reinterpret_cast<float*>(after_k + (cache_norm ? (size_t)0 : (size_t)nq16 * KROW));  // [W][cols] (bf16)
+    float* colsum = reinterpret_cast<float*>(after_k + ((cache_norm || guide_global) ? (size_t)0 : (size_t)nq16 * KROW));  // [W][cols] (bf16)
     const int wstride = D + n_stage + cols;
     float* wbuf = reinterpret_cast<float*>(after_k);                            // [W][D + n_stage + cols]   (fp32)
     float* S = kMma ? colsum + W * cols : wbuf + W * wstride;
@@ -287,7 +289,7 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
     const T* gq = reinterpret_cast<const T*>(lv.guide) + (size_t)unit * nq * D;
     if constexpr (kMma) {
         // ---- Eq. 9 on tensor cores: stage the guide rows (mid-only scoring), clear the column sums
-        if (!cache_norm) {
+        if (!cache_norm && !guide_global) {
             for (int idx = tid; idx < nq16 * CHUNKS; idx += blockDim.x) {
                 const int r = idx / CHUNKS, c = idx - r * CHUNKS;
                 uint4 val = make_uint4(0u, 0u, 0u, 0u);
@@ -299,6 +301,8 @@ __global__ void __launch_bounds__(1024) line_end_kernel(const LayerView lv0, con
         __syncthreads();
         if (cache_norm)
             score_mma<D, true>(kst, qg, reinterpret_cast<const uint32_t*>(gq), colsum, n_stage, col_off, cols, nq, G, n, scale_log2, warp, lane, W);
+        else if (guide_global)
+            score_mma<D, false, true>(kst, qg, reinterpret_cast<const uint32_t*>(gq), colsum, n_stage, col_off, cols, nq, G, n, scale_log2, warp, lane, W);
         else
             score_mma<D, false>(kst, qg, nullptr, colsum, n_stage, col_off, cols, nq, G, n, scale_log2, warp, lane, W);
         __syncthreads();

@@ -113,6 +113,17 @@ def test_struct_size_is_checked_and_null_arguments():
     assert L.lar_cache_launch_count(None) == 0
 
 
+def test_a_mid_region_too_large_to_stage_with_the_guide_rows_still_gets_a_plan():
+    """1024-px shape at a quarter of the tokens: 520 mid keys + 260 guide rows of 272 B exceed 227 KB; the plan then reads
+    the guide rows from global memory (8 warps) instead of refusing the configuration."""
+    w = W.WORKLOADS["gqa_1024"]
+    quarter = w.scaled(budget_lines=16, recent_lines=7, anchor_len=w.line_width)
+    assert quarter.mid_len == 520
+    p = lar.lar_plan_query(lar.config_from_workload(quarter))
+    assert 520 * 272 < p.line_end_smem_bytes <= 227 * 1024
+    assert p.line_end_smem_bytes < lar.lar_plan_query(lar.config_from_workload(w.scaled(budget_lines=12, recent_lines=5))).line_end_smem_bytes
+
+
 def test_full_cache_budget_and_overrides():
     p = lar.lar_plan_query(_cfg(budget_lines=8))
     assert p.compressing == 0 and p.capacity == 4 + 64

@@ -172,6 +172,8 @@ QUOTED = {
     "llamagen_xl budget 6 lines (1/4)": lambda: _with_budget(W.WORKLOADS["llamagen_xl"], 6),
     "lumina_768 budget 12 lines (1/4)": lambda: _with_budget(W.WORKLOADS["lumina_768"], 12),
     "lumina_768 budget 8 lines (1/6)": lambda: _with_budget(W.WORKLOADS["lumina_768"], 8),
+    # M = 520 mid keys and 260 guide rows do not fit into shared memory together: the guide rows are read from global
+    "gqa_1024 budget 16 lines (1/4)": lambda: _with_budget(W.WORKLOADS["gqa_1024"], 16),
 }
 
 
