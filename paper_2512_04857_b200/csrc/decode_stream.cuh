@@ -214,7 +214,10 @@ __device__ __forceinline__ int range_owner(int t, int n, int P) {
     return t < head ? t / (q + 1) : r + (t - head) / q;
 }
 
-template <int D, int G>
+// VIEWS: q / k / v / out may be views of larger tensors (the *_seq_stride arguments) and the rotary embedding of q and
+// the new k may be fused in (a.rope, a.rope_mode); a kernel of its own, so that launches on dense tensors carry none of
+// that per-segment work (with many short units per CTA the epilogue warp's work per unit sets the pace)
+template <int D, int G, bool VIEWS>
 __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs a, const __grid_constant__ TensorMaps tm) {
     using TR = MmaTraits<D>;
     using T16 = __nv_bfloat16;
@@ -244,7 +247,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     const uint32_t bar_pfull = bar_qempty + kMaxQSlots * 8, bar_pempty = bar_pfull + 2 * 8;
     const uint32_t bar_qrot = bar_pempty + 2 * 8;  // (rotary embedding) the slot's q and k rows have been rotated
     // what the consumers wait for before they take a segment's queries
-    const uint32_t bar_qready = a.rope_mode ? bar_qrot : bar_qfull;
+    const uint32_t bar_qready = (VIEWS && a.rope_mode) ? bar_qrot : bar_qfull;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_ptr + (2 * NS + 3 * kMaxQSlots + 4) * 8);
 
     // Dependents may be scheduled from now on: they only hint the L2 before their own griddepcontrol.wait, and a
@@ -301,7 +304,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     // producer's first K/V copies are not queued behind them.
     // element offset of unit `u`'s rows in a [sequence][head][d] tensor with `per_head` elements per KV head
     auto unit_offset = [&](int u, long long seq_stride, int per_head) -> size_t {
-        if (seq_stride == 0) return (size_t)u * per_head;
+        if (!VIEWS || seq_stride == 0) return (size_t)u * per_head;
         const int sq = u / lv.n_kv_heads;
         return (size_t)sq * (size_t)seq_stride + (size_t)(u - sq * lv.n_kv_heads) * per_head;
     };
@@ -626,7 +629,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             // rotary embedding: cos and sin of this sequence's position for the pairs this lane rotates (on their way
             // while the inputs arrive)
             float rc[D / 64], rs[D / 64];
-            if (a.rope_mode) {
+            if (VIEWS && a.rope_mode) {
                 const float* cs = a.rope + (size_t)(unit / lv.n_kv_heads) * D;
 #pragma unroll
                 for (int k = 0; k < D / 64; ++k) {
@@ -638,7 +641,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             const unsigned char* Qs = qring_ptr + qs * QENT;
             const uint16_t* Q16 = reinterpret_cast<const uint16_t*>(Qs);
-            if (a.rope_mode) {
+            if (VIEWS && a.rope_mode) {
                 // q (all G heads) and the new k row are rotated in place, pair by pair, in fp32 with every product and
                 // sum rounded separately, then rounded to bf16: the cache, the guide queue and the logits see rotated rows
                 T16* rows = reinterpret_cast<T16*>(qring_ptr + qs * QENT);

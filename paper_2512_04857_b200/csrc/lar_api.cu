@@ -398,18 +398,20 @@ lar_status_t make_tensor_maps(lar_cache* c) {
 
 // ---- kernel tables ------------------------------------------------------------------------------
 using DecodeStreamFn = void (*)(const lar::StreamArgs, const lar::TensorMaps);
-template <int D>
+template <int D, bool VIEWS>
 DecodeStreamFn decode_stream_for_group(int G) {
     switch (G) {
-        case 1: return lar::decode_stream_kernel<D, 1>;
-        case 2: return lar::decode_stream_kernel<D, 2>;
-        case 4: return lar::decode_stream_kernel<D, 4>;
-        case 8: return lar::decode_stream_kernel<D, 8>;
+        case 1: return lar::decode_stream_kernel<D, 1, VIEWS>;
+        case 2: return lar::decode_stream_kernel<D, 2, VIEWS>;
+        case 4: return lar::decode_stream_kernel<D, 4, VIEWS>;
+        case 8: return lar::decode_stream_kernel<D, 8, VIEWS>;
     }
     return nullptr;
 }
-DecodeStreamFn decode_stream_fn(const lar_config_t& c, int G) {
-    return c.head_dim == 64 ? decode_stream_for_group<64>(G) : decode_stream_for_group<128>(G);
+// views: q / k / v / out with sequence strides and / or the rotary embedding fused in
+DecodeStreamFn decode_stream_fn(const lar_config_t& c, int G, bool views = false) {
+    if (views) return c.head_dim == 64 ? decode_stream_for_group<64, true>(G) : decode_stream_for_group<128, true>(G);
+    return c.head_dim == 64 ? decode_stream_for_group<64, false>(G) : decode_stream_for_group<128, false>(G);
 }
 using DecodeFn = void (*)(const lar::DecodeArgs);
 using LineEndFn = void (*)(const lar::LayerView, const lar::LayerStrides, float, int);
@@ -540,7 +542,7 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
         lc.blockDim = dim3((unsigned)(32 * (c->plan.warps_per_cta + lar::kProducers + 1)), 1, 1);
         lc.attrs = attrs;
         lc.numAttrs = na;
-        DecodeStreamFn fn = decode_stream_fn(c->cfg, c->d.group);
+        DecodeStreamFn fn = decode_stream_fn(c->cfg, c->d.group, ss.rope_mode != 0 || ss.q || ss.k || ss.v || ss.out);
         LAR_CUDA(cudaLaunchKernelEx(&lc, fn, a, c->tmaps));
     } else {
         if (ss.q || ss.k || ss.v || ss.out || ss.rope) return LAR_ERR_INVALID_ARG;  // fp32 storage: dense tensors only
@@ -675,6 +677,9 @@ lar_status_t lar_cache_create(const lar_config_t* cfg, void* dev_slab, size_t sl
     if (ce == cudaSuccess)
         ce = cudaFuncSetAttribute(cfg->dtype == LAR_BF16 ? (const void*)decode_stream_fn(*cfg, d.group) : (const void*)decode_fn(*cfg, d.group),
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, plan.decode_smem_bytes);
+    if (ce == cudaSuccess && cfg->dtype == LAR_BF16)  // (the variant for views of larger tensors / the rotary embedding)
+        ce = cudaFuncSetAttribute((const void*)decode_stream_fn(*cfg, d.group, true), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  plan.decode_smem_bytes);
     if (ce == cudaSuccess && d.compressing)
         ce = cudaFuncSetAttribute((const void*)line_end_fn(*cfg, d.group), cudaFuncAttributeMaxDynamicSharedMemorySize, plan.line_end_smem_bytes);
     if (ce == cudaSuccess) ce = cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking);
