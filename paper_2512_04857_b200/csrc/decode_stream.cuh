@@ -144,6 +144,7 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {
 
 // ---- shared-memory plan of decode_stream_kernel (host and device agree through these) -------------
 constexpr int kMaxConsumers = 6;  // consumer warps per CTA at most
+constexpr int kPartialPad = 4;    // floats behind the D values of a partial: m, l and padding that keeps rows 16-byte aligned
 constexpr int kProducers = 2;     // producer warps per CTA: tile j is fetched by producer j % kProducers
 constexpr int kMaxQSlots = 8;     // depth of the query ring at most
 // query ring / partial buffers of a CTA that works on at most `segs` segments per launch
@@ -159,7 +160,7 @@ __host__ __device__ constexpr int stream_q_entry_bytes(int D, int G) { return ((
 __host__ __device__ constexpr int stream_fixed_smem_bytes(int D, int G, int W, int NQ, int NPB) {
     return 1024                                  // slack: the ring starts on a 1024-byte boundary
            + NQ * stream_q_entry_bytes(D, G)     // query ring
-           + NPB * (W + 1) * G * (D + 2) * 4     // partial buffers
+           + NPB * (W + 1) * G * (D + kPartialPad) * 4  // partial buffers
            + (3 * kMaxQSlots + 4) * 8 + 16;      // query / partial barriers, abort flag
 }
 __host__ __device__ constexpr int stream_smem_bytes(int D, int G, int W, int NS, int NQ, int NPB) {
@@ -224,7 +225,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     const int NQ = a.q_slots, NPB = a.p_bufs;  // powers of two
     const int qsh = __ffs(NQ) - 1, psh = NPB - 1;
     constexpr int QENT = stream_q_entry_bytes(D, G);
-    constexpr int PS = D + 2;  // floats per (warp, head) partial: o[D], m, l
+    constexpr int PS = D + kPartialPad;  // floats per (warp, head) partial: o[D], m, l (+ padding: 16-byte aligned rows)
     constexpr int PER = D / 32;
     extern __shared__ unsigned char smem_raw[];
 
@@ -604,7 +605,9 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         T16* outp = reinterpret_cast<T16*>(a.out);
         // What closing a unit needs from global memory (the page that takes the new row, the unit's length
         // in device memory) is requested one segment ahead, so that its latency never stalls this warp.
-        const int new_page_idx = len / lv.page_tokens;
+        const int new_page_idx = len / lv.page_tokens, new_row_in_page = len - new_page_idx * lv.page_tokens;
+        const int step_tok = a.fused ? n_tok : n_tok - 1;  // 0-based visual index of this step's token
+        const int guide_slot = step_tok >= 0 ? step_tok % lv.line_width : 0;
         auto closing_loads = [&](int sg, int& page, int& dev_len) {
             const int un = u0 + sg;
             page = 0;
@@ -662,10 +665,12 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             }
 
             // ---- the token of this step (Eq. 4, 8): logit per head, value row, stores
-            // Merge layout: the warp's lanes are split over the G heads, LPH lanes per head; lane (hg, sub) owns the
-            // elements sub, sub + LPH, ... of head hg (EPH of them) -- one set of exponentials per lane, not G.
+            // Merge layout: the warp's lanes are split over the G heads, LPH lanes per head; lane (hg, sub) owns the EPH
+            // consecutive elements from e0 = sub * EPH of head hg (vector loads from the partials, one vector store of the
+            // output) -- one set of exponentials per lane, not G.
             constexpr int LPH = 32 / G, EPH = D / LPH;
-            const int hg = lane / LPH, sub = lane % LPH;
+            constexpr int VEC = EPH % 4 == 0 ? 4 : 2;  // floats per shared-memory load
+            const int hg = lane / LPH, sub = lane % LPH, e0 = sub * EPH;
             float s_new[G], v_new[EPH];
             const bool with_new = a.fused && closes;
 #pragma unroll
@@ -680,7 +685,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
 #pragma unroll
                     for (int i = 0; i < PER; ++i) kf[i] = bf16_bits_to_float(K16[lane + 32 * i]);
 #pragma unroll
-                    for (int i = 0; i < EPH; ++i) v_new[i] = bf16_bits_to_float(V16[sub + LPH * i]);
+                    for (int i = 0; i < EPH; ++i) v_new[i] = bf16_bits_to_float(V16[e0 + i]);
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
                         float sv = 0.f;
@@ -691,7 +696,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                         s_new[g] = sv * a.scale_log2;
                     }
                     if (len < lv.cap) {
-                        const size_t off = ((size_t)page_cur * lv.page_tokens + len % lv.page_tokens) * TR::ROW_BYTES;
+                        const size_t off = ((size_t)page_cur * lv.page_tokens + new_row_in_page) * TR::ROW_BYTES;
                         const uint32_t* K32 = reinterpret_cast<const uint32_t*>(K16);
                         const uint32_t* V32 = reinterpret_cast<const uint32_t*>(V16);
                         for (int i = lane; i < D / 2; i += 32) {
@@ -715,11 +720,9 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                     }
                 }
                 // Eq. 8: the queries join the guide queue of the line being generated
-                const int tok = a.fused ? n_tok : n_tok - 1;  // 0-based visual index of this step's token
-                if (tok >= 0) {
-                    const int slot = tok % lv.line_width;
+                if (step_tok >= 0) {
                     uint32_t* gq = reinterpret_cast<uint32_t*>(reinterpret_cast<T16*>(lv.guide) +
-                                                               (((size_t)unit * lv.line_width + slot) * G) * D);
+                                                               (((size_t)unit * lv.line_width + guide_slot) * G) * D);
                     const uint32_t* Q32 = reinterpret_cast<const uint32_t*>(Qs);
                     for (int i = lane; i < G * D / 2; i += 32) gq[i] = Q32[i];
                 }
@@ -755,7 +758,18 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                     const float f = exp2_or_zero(mw[w], M);
                     L = fmaf(pw[D + 1], f, L);
 #pragma unroll
-                    for (int i = 0; i < EPH; ++i) Oh[i] = fmaf(pw[sub + LPH * i], f, Oh[i]);
+                    for (int i = 0; i < EPH; i += VEC) {
+                        float t[4];
+                        if constexpr (VEC == 4) {
+                            const float4 x = *reinterpret_cast<const float4*>(pw + e0 + i);
+                            t[0] = x.x; t[1] = x.y; t[2] = x.z; t[3] = x.w;
+                        } else {
+                            const float2 x = *reinterpret_cast<const float2*>(pw + e0 + i);
+                            t[0] = x.x; t[1] = x.y;
+                        }
+#pragma unroll
+                        for (int k = 0; k < VEC; ++k) Oh[i + k] = fmaf(t[k], f, Oh[i + k]);
+                    }
                 }
                 Mh = M;
                 Lh = L;
@@ -769,9 +783,19 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             if (opens && closes) {
                 // the whole unit lies in this CTA
                 const float inv = Lh > 0.f ? 1.f / Lh : 0.f;
+                uint32_t packed[EPH / 2];
 #pragma unroll
-                for (int i = 0; i < EPH; ++i)
-                    outp[out_base + (size_t)hg * D + sub + LPH * i] = __float2bfloat16_rn(Oh[i] * inv);
+                for (int i = 0; i < EPH / 2; ++i) packed[i] = pack_bf16(Oh[2 * i] * inv, Oh[2 * i + 1] * inv);
+                T16* dst = outp + out_base + (size_t)hg * D + e0;  // EPH * 2 bytes, aligned to their size (up to 16)
+                if constexpr (EPH % 8 == 0) {
+#pragma unroll
+                    for (int i = 0; i < EPH / 8; ++i)
+                        reinterpret_cast<uint4*>(dst)[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+                } else if constexpr (EPH == 4) {
+                    *reinterpret_cast<uint2*>(dst) = make_uint2(packed[0], packed[1]);
+                } else {
+                    *reinterpret_cast<uint32_t*>(dst) = packed[0];
+                }
             } else {
                 // the unit is shared with neighbouring CTAs: leave a partial, the last one to arrive merges
                 const int p_first = range_owner(ub, total, Pe);
@@ -782,7 +806,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                 }
                 float* mine = a.partials + ((size_t)unit * a.max_seg + (p - p_first)) * G * PS;
 #pragma unroll
-                for (int i = 0; i < EPH; ++i) mine[hg * PS + sub + LPH * i] = Oh[i];
+                for (int i = 0; i < EPH; ++i) mine[hg * PS + e0 + i] = Oh[i];
                 if (sub == 0) {
                     mine[hg * PS + D] = Mh;
                     mine[hg * PS + D + 1] = Lh;

@@ -194,7 +194,7 @@ void make_layout(const lar_config_t* c, const Derived& d, Layout& L) {
     L.stride_pool = align_up(U * d.ppu * d.P * d.row_bytes, 256);
     L.off_kpool = take(L.stride_pool * Lyr);
     L.off_vpool = take(L.stride_pool * Lyr);
-    L.off_partials = take(c->dtype == LAR_BF16 ? U * d.max_seg * d.group * (c->head_dim + 2) * sizeof(float) : 0);
+    L.off_partials = take(c->dtype == LAR_BF16 ? U * d.max_seg * d.group * (c->head_dim + lar::kPartialPad) * sizeof(float) : 0);
     L.tickets_bytes = U * sizeof(int);  // one ticket per unit
     L.off_tickets = take(L.tickets_bytes);
     L.total = off;
