@@ -64,6 +64,11 @@ struct StreamArgs {
     int fused;          // 1: the step's token comes from k_new / v_new and is appended by this kernel
     int prefetch;       // 1: the CTA may fill its ring before waiting for the preceding kernel (units whose length is published)
     int n_units, n_stages, max_seg;
+    // what the host knows about the launch's tile list, so that a CTA divides nothing on its way to its first copy:
+    int tiles_per_unit;        // T = ceil(len / 32), 1 for an empty cache
+    unsigned tiles_magic;      // floor(2^32 / T) + 1: x / T = umulhi(x, magic) up to a correction of one
+    int range_ctas, range_q, range_r;  // CTAs that get work, items per CTA, CTAs that get one item more (items: units or tiles)
+    int page_shift;            // log2(page_tokens)
     int seq, need_seq;  // sequence number of this launch on its cache / of the launch that last wrote this layer's cache
     int* done_seq;      // device word: every launch up to this number has completed
     int q_slots, p_bufs;  // depth of the CTA's query ring / number of partial buffers
@@ -184,6 +189,15 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
     }
     return true;
 }
+// barrier initialisations become visible to the copy engine's arrivals (shared memory only: nothing in flight to
+// global memory is waited for)
+__device__ __forceinline__ void mbar_fence_init_smem() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+// named CTA barriers: `threads` threads take part; arrive does not wait
+__device__ __forceinline__ void named_bar_sync(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
+__device__ __forceinline__ void named_bar_arrive(int id, int threads) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -232,7 +246,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int W = (int)(blockDim.x >> 5) - kProducers - 1;  // consumer warps
     const int NS = a.n_stages;
-    const int P = (int)gridDim.x, p = (int)blockIdx.x;
+    const int p = (int)blockIdx.x;
     const LayerView& lv = a.lv;
 
     const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -254,51 +268,62 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     // Dependents may be scheduled from now on: they only hint the L2 before their own griddepcontrol.wait, and a
     // dependent's wait covers this whole grid (which itself waits for its predecessor below).
     grid_dep_launch();
+    // the completion word of the cache (see the producers): requested first, it is needed a microsecond from now
+    int done_seq_seen = 0;
+    if (warp < kProducers && a.prefetch) done_seq_seen = ld_acquire_gpu(a.done_seq);
 
-    {
-        // one barrier per thread (the set-up of a launch is on the path between two launches)
-        const int t = (int)threadIdx.x;
-        if (t < 2 * NS) {
-            mbar_init(bar_full + t * 8, 1);  // full / empty of the K/V ring (adjacent in memory)
-        } else if (t < 2 * NS + NQ) {
-            mbar_init(bar_qfull + (t - 2 * NS) * 8, 1);
-        } else if (t < 2 * NS + 2 * NQ) {
-            mbar_init(bar_qempty + (t - 2 * NS - NQ) * 8, (uint32_t)(W + 1));
-        } else if (t < 2 * NS + 2 * NQ + 2) {
-            mbar_init(bar_pfull + (t - 2 * NS - 2 * NQ) * 8, (uint32_t)W);
-        } else if (t < 2 * NS + 2 * NQ + 4) {
-            mbar_init(bar_pempty + (t - 2 * NS - 2 * NQ - 2) * 8, 1);
-        } else if (t < 2 * NS + 3 * NQ + 4) {
-            mbar_init(bar_qrot + (t - 2 * NS - 2 * NQ - 4) * 8, 1);
+    // The set-up of a launch is on the path between two launches: the two producer warps initialise every barrier (each
+    // thread one or two), agree among themselves, tell the other warps without waiting for them (bar.arrive) and go on
+    // to their first copies; the other warps wait for that signal only.
+    if (warp < kProducers) {
+        const int n_bars = 2 * NS + 3 * NQ + 4;
+        for (int t = (int)threadIdx.x; t < n_bars; t += kProducers * 32) {
+            if (t < 2 * NS) {
+                mbar_init(bar_full + t * 8, 1);  // full / empty of the K/V ring (adjacent in memory)
+            } else if (t < 2 * NS + NQ) {
+                mbar_init(bar_qfull + (t - 2 * NS) * 8, 1);
+            } else if (t < 2 * NS + 2 * NQ) {
+                mbar_init(bar_qempty + (t - 2 * NS - NQ) * 8, (uint32_t)(W + 1));
+            } else if (t < 2 * NS + 2 * NQ + 2) {
+                mbar_init(bar_pfull + (t - 2 * NS - 2 * NQ) * 8, (uint32_t)W);
+            } else if (t < 2 * NS + 2 * NQ + 4) {
+                mbar_init(bar_pempty + (t - 2 * NS - 2 * NQ - 2) * 8, 1);
+            } else {
+                mbar_init(bar_qrot + (t - 2 * NS - 2 * NQ - 4) * 8, 1);
+            }
         }
-        if (t == 0) *abort_flag = 0;
-        if (t < 2 * NS + 3 * NQ + 4) mbar_fence_init();
+        if (threadIdx.x == 0) *abort_flag = 0;
+        mbar_fence_init_smem();
+        named_bar_sync(2, kProducers * 32);
+        named_bar_arrive(1, (int)blockDim.x);
+    } else {
+        named_bar_sync(1, (int)blockDim.x);
     }
-    __syncthreads();
 
 
     // ---- the layer's tile list and this CTA's range of it
     const int len = a.len, n_tok = a.n_tok;
-    const int T = len > 0 ? (len + kStreamTile - 1) / kStreamTile : 1;  // an empty cache is one tile of 0 rows
+    const int T = a.tiles_per_unit;  // ceil(len / 32); an empty cache is one tile of 0 rows
     const int total = a.n_units * T;
+    // x / T for 0 <= x < 2^30 without a division (the host's multiplier, corrected by at most one)
+    auto div_T = [&](int x) {
+        if (T == 1) return x;  // (the multiplier of 1 does not fit 32 bits)
+        int q = (int)__umulhi((unsigned)x, a.tiles_magic);
+        if (q * T > x) --q;
+        else if ((q + 1) * T <= x) ++q;
+        return q;
+    };
     int t_begin = 0, t_end = 0;
-    int Pe;  // CTAs that get work: every range is non-empty
-    if (a.unit_ranges) {
-        Pe = a.n_units < P ? a.n_units : P;
-        if (p < Pe) {
-            t_begin = range_begin(a.n_units, Pe, p) * T;
-            t_end = range_begin(a.n_units, Pe, p + 1) * T;
-        }
-    } else {
-        Pe = total < P ? total : P;
-        if (p < Pe) {
-            t_begin = range_begin(total, Pe, p);
-            t_end = range_begin(total, Pe, p + 1);
-        }
+    const int Pe = a.range_ctas;  // CTAs that get work: every range is non-empty
+    if (p < Pe) {
+        // the first range_r CTAs get range_q + 1 items, the others range_q (items: whole units, or tiles)
+        const int b0 = p * a.range_q + (p < a.range_r ? p : a.range_r), b1 = b0 + a.range_q + (p < a.range_r ? 1 : 0);
+        t_begin = a.unit_ranges ? b0 * T : b0;
+        t_end = a.unit_ranges ? b1 * T : b1;
     }
     const int n_tiles = t_end - t_begin;
-    const int u0 = t_begin / T;
-    const int n_segs = n_tiles > 0 ? (t_end - 1) / T - u0 + 1 : 0;
+    const int u0 = div_T(t_begin);
+    const int n_segs = n_tiles > 0 ? div_T(t_end - 1) - u0 + 1 : 0;
 
     // One lane requests the inputs of segment `seg`: its queries and, where the segment closes its unit in a fused
     // step, the new k and v rows.  Issued by the epilogue warp, which is idle when a launch starts, so that the
@@ -337,7 +362,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         // launches up to that one have completed and their writes are visible to it).  The rows of this layer are
         // final once the launch that last wrote them (need_seq, from the host) is covered by that word.
         int fill_end = 0;
-        if (a.prefetch && ld_acquire_gpu(a.done_seq) >= a.need_seq) {
+        if (a.prefetch && done_seq_seen >= a.need_seq) {
             fence_proxy_async_global();  // the copies below read what the acquire made visible
             fill_end = n_tiles < NS ? n_tiles : NS;
         }
@@ -346,14 +371,14 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
 
         auto describe = [&](int jj, int& y, int& rows, int& tile) {
             const int t = t_begin + jj;
-            const int unit = t / T;
+            const int unit = div_T(t);
             tile = t - unit * T;
             const int row0 = tile * kStreamTile;
             rows = len - row0 < kStreamTile ? len - row0 : kStreamTile;
             if (rows > 0) {
-                const int pidx = unit * lv.pages_per_unit + row0 / lv.page_tokens;
+                const int pidx = unit * lv.pages_per_unit + (row0 >> a.page_shift);
                 const int page = lv.identity_pages ? pidx : __ldg(&lv.page_table[pidx]);
-                y = a.pool_row_base + page * lv.page_tokens + row0 % lv.page_tokens;
+                y = a.pool_row_base + (page << a.page_shift) + (row0 & (lv.page_tokens - 1));
             } else {
                 y = 0;
             }

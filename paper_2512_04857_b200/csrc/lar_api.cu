@@ -519,6 +519,20 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
             a.n_tok = sh.n_tok;
         }
         a.unit_ranges = c->d.unit_ranges;
+        {
+            // the launch's tile list: T tiles per unit; the CTAs' ranges are whole units or tiles
+            const int T = a.len > 0 ? (a.len + lar::kStreamTile - 1) / lar::kStreamTile : 1;
+            const long long items = c->d.unit_ranges ? (long long)c->d.units : (long long)c->d.units * T;
+            const int pe = (int)(items < c->d.ctas ? items : c->d.ctas);
+            a.tiles_per_unit = T;
+            a.tiles_magic = (unsigned)((1ull << 32) / (unsigned)T + 1ull);
+            a.range_ctas = pe;
+            a.range_q = (int)(items / pe);
+            a.range_r = (int)(items % pe);
+            int sh = 0;
+            while ((1 << sh) < c->d.P) ++sh;
+            a.page_shift = sh;
+        }
         a.scale_log2 = scale_log2;
         a.fused = fused;
         a.prefetch = prefetch;
