@@ -62,7 +62,8 @@ struct StreamArgs {
     const float* rope;  // rotary embedding: [sequence][d] floats, cos of the d/2 pairs then sin, for this step's position
     int rope_mode;      // 0: none; 1: pairs (i, i + d/2); 2: pairs (2 i, 2 i + 1)
     int fused;          // 1: the step's token comes from k_new / v_new and is appended by this kernel
-    int prefetch;       // 1: the CTA may fill its ring before waiting for the preceding kernel (units whose length is published)
+    int prefetch;       // the CTA may fill its ring before waiting for the preceding kernel: 1 if the completion word covers
+                        // need_seq; 2 unconditionally (the host knows that launch need_seq cannot be in flight any more)
     int n_units, n_stages, max_seg;
     // what the host knows about the launch's tile list, so that a CTA divides nothing on its way to its first copy:
     int tiles_per_unit;        // T = ceil(len / 32), 1 for an empty cache
@@ -268,9 +269,6 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
     // Dependents may be scheduled from now on: they only hint the L2 before their own griddepcontrol.wait, and a
     // dependent's wait covers this whole grid (which itself waits for its predecessor below).
     grid_dep_launch();
-    // the completion word of the cache (see the producers): requested first, it is needed a microsecond from now
-    int done_seq_seen = 0;
-    if (warp < kProducers && a.prefetch) done_seq_seen = ld_acquire_gpu(a.done_seq);
 
     // The set-up of a launch is on the path between two launches: the two producer warps initialise every barrier (each
     // thread one or two), agree among themselves, tell the other warps without waiting for them (bar.arrive) and go on
@@ -360,9 +358,11 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
         // ---- before the dependency: may the ring be filled already?  Every launch on a cache carries a sequence
         // number; a decode kernel whose own dependency has resolved publishes the number of its predecessor (all
         // launches up to that one have completed and their writes are visible to it).  The rows of this layer are
-        // final once the launch that last wrote them (need_seq, from the host) is covered by that word.
+        // final once the launch that last wrote them (need_seq, from the host) is covered by that word -- or, without
+        // looking, if that launch lies further back than launches can be in flight at all (the host's bound: every
+        // launch but the oldest in flight is wholly resident, waiting for its predecessor).
         int fill_end = 0;
-        if (a.prefetch && done_seq_seen >= a.need_seq) {
+        if (a.prefetch == 2 || (a.prefetch == 1 && ld_acquire_gpu(a.done_seq) >= a.need_seq)) {
             fence_proxy_async_global();  // the copies below read what the acquire made visible
             fill_end = n_tiles < NS ? n_tiles : NS;
         }

@@ -301,6 +301,7 @@ struct lar_cache {
     Layout L;
     char* slab;
     int device;
+    int sm_count;  // SMs of that device
     bool host_checks;
     float scale;
     uint64_t launches;
@@ -541,6 +542,15 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
         a.max_seg = c->d.max_seg;
         a.seq = ++c->seq;
         a.need_seq = c->last_writer[layer];
+        if (prefetch) {
+            // How far back can a launch of this cache still be in flight?  A decode kernel lets its successor start at once
+            // and leaves only after its predecessor has completed, so every launch in flight but the oldest holds all its
+            // CTAs: with `slots` CTAs of this size resident on the GPU at most, the oldest is (slots - 1) / ctas + 1 back.
+            const long long per_sm = 233472 / ((long long)c->plan.decode_smem_bytes + 1024);
+            const long long slots = (long long)c->sm_count * (per_sm < 1 ? 1 : per_sm > 32 ? 32 : per_sm);
+            const long long depth = (slots - 1) / c->d.ctas + 1;
+            if ((long long)a.seq - a.need_seq > depth + 1) a.prefetch = 2;  // (one launch of margin)
+        }
         c->last_writer[layer] = a.seq;
         a.done_seq = reinterpret_cast<int*>(c->slab + c->L.off_status + 128);
         a.q_slots = c->d.q_slots;
@@ -660,6 +670,7 @@ lar_status_t lar_cache_create(const lar_config_t* cfg, void* dev_slab, size_t sl
 
     auto fail = [&](lar_status_t e) { delete c; return e; };
     cudaError_t ce = cudaGetDevice(&c->device);
+    if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
     if (ce != cudaSuccess) { g_last_cuda_error = (int)ce; return fail(LAR_ERR_CUDA); }
 
     // page tables: unit u owns pages_per_unit pages of its layer's pool (identity, or shuffled)
