@@ -384,8 +384,7 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             }
         };
         // Lane 0 issues; all lanes look the page ids of a batch of 32 tiles up together, one batch ahead.
-        // Stage and phase advance incrementally (no division in the per-tile path).  A fresh mbarrier lets a
-        // wait on parity 1 pass, so the first trip round the ring does not wait for the consumers.
+        // Stage and phase advance incrementally (no division in the per-tile path).
         int y_n = 0, rt_n = 0;  // rt = rows | tile << 8
         {
             int r = 0, t = 0;
@@ -412,7 +411,8 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                 const int yi = __shfl_sync(0xffffffffu, y, i), rti = __shfl_sync(0xffffffffu, rt, i);
                 if (lane == 0 && ok) {
                     const int ri = rti & 0xff;
-                    ok = wait_or_abort(bar_empty + stage * 8, empty_parity, abort_flag);
+                    // (the first trip round the ring finds every stage free: no wait on the way to the first copies)
+                    if (i0 + i >= NS / kProducers) ok = wait_or_abort(bar_empty + stage * 8, empty_parity, abort_flag);
                     if (ok) {
                         const uint32_t bar = bar_full + stage * 8, dst = ring + (uint32_t)stage * TR::STAGE_BYTES;
                         if (ri > 0) {
