@@ -449,12 +449,28 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             const int ub = unit * T;
             const int je = (ub + T < t_end ? ub + T : t_end) - t_begin;
 
-            // ---- Q fragments (A operand): row qrow = head, 16 columns per k-step; heads >= G are zero rows
+            // ---- Q fragments (B operand): column qrow = head, 16 dims per k-step; heads >= G are zero columns
             const int qs = seg & (NQ - 1);
-            ok = wait_or_abort(bar_qready + qs * 8, (uint32_t)(((seg >> qsh)) & 1), abort_flag);
-            if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+            // The queries of the CTA's first unit are what the whole launch waits for once its dependency has resolved:
+            // the consumers read them straight from global memory (L2: hinted there before the wait), which is quicker
+            // than waiting for the epilogue warp's copy into shared memory and its barrier.  (Not with the fused rotary
+            // embedding: the rotated rows exist in shared memory only.)
+            const bool q_direct = seg == 0 && !(VIEWS && a.rope_mode);
             uint32_t qa0[TR::KSTEPS], qa2[TR::KSTEPS];
-            {
+            if (q_direct) {
+                const uint32_t* Qg = reinterpret_cast<const uint32_t*>(reinterpret_cast<const T16*>(a.q) + unit_offset(unit, a.q_seq_stride, G * D));
+#pragma unroll
+                for (int s = 0; s < TR::KSTEPS; ++s) {
+                    qa0[s] = 0u;
+                    qa2[s] = 0u;
+                    if (qrow < G) {
+                        qa0[s] = __ldcg(Qg + (qrow * D + 16 * s + 2 * quad) / 2);
+                        qa2[s] = __ldcg(Qg + (qrow * D + 16 * s + 8 + 2 * quad) / 2);
+                    }
+                }
+            } else {
+                ok = wait_or_abort(bar_qready + qs * 8, (uint32_t)(((seg >> qsh)) & 1), abort_flag);
+                if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
                 const unsigned char* Qs = qring_ptr + qs * QENT;
 #pragma unroll
                 for (int s = 0; s < TR::KSTEPS; ++s) {
@@ -465,9 +481,9 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                         qa2[s] = *reinterpret_cast<const uint32_t*>(Qs + (qrow * D + 16 * s + 8 + 2 * quad) * 2);
                     }
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_qempty + qs * 8);
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_qempty + qs * 8);
 
             // running maximum and this thread's share of the row sum of heads 2 quad and 2 quad + 1
             float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
@@ -565,6 +581,13 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
                 if (lane == 0) mbar_arrive(bar_empty + s * 8);
             }
             if (!ok) break;
+            if (q_direct) {
+                // the slot of the first segment is released here, after its copy has landed (long ago: a waiter must
+                // have seen every phase of a barrier it will wait on again)
+                ok = wait_or_abort(bar_qready + qs * 8, 0u, abort_flag);
+                if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+                if (lane == 0) mbar_arrive(bar_qempty + qs * 8);
+            }
 
             // ---- this warp's partial of the segment -> shared memory
             const int buf = seg & (NPB - 1);
