@@ -31,7 +31,7 @@ UNIT = "image_tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch (bytes), from an ncu capture of a 4-layer case of
 # the same shape and launch configuration (one launch = one layer, so the capture gives the per-launch figure of the
 # full workload); null for shapes that have no capture
-NCU_TRAFFIC_PER_LAUNCH = {"janus_pro_7b": 78.2e6, "gqa_1024": 42.4e6, "llamagen_xl": 26.8e6}
+NCU_TRAFFIC_PER_LAUNCH = {"janus_pro_7b": 78.0e6, "gqa_1024": 42.4e6, "llamagen_xl": 26.8e6}
 
 
 def max_over_ranks(values, dist, device):
