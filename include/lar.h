@@ -91,6 +91,12 @@ typedef enum { LAR_BF16 = 0, LAR_FP32 = 1 } lar_dtype_t;
                                         (the index map is not monotone); the line end finds the mid region of Sec. 3.3
                                         through the index map.  Kept sets, outputs and scores are unchanged. */
 
+#define LAR_FLAG_TEST_STALL 0x100u    /* test hook for the bounded waits of the bf16 decode kernel: its producer warps request no
+                                        K/V tile, so every consumer warp's wait for its first tile runs into the limit
+                                        (~1 s of SM clocks); the CTA's roles then give up, the launch ends by itself after
+                                        1-3 s, outputs are undefined and status bit 4 (wait limit) is recorded.  The
+                                        device and the slab stay usable.  No counterpart in the paper. */
+
 #define LAR_FLAG_HOST_DEFER_OUT 0x20u /* lar_decode_step_host does not make `stream` wait for its copy-out: the
                                         copy-out of a call then overlaps the kernels of the next calls as well.
                                         `out_host` of a call is complete only after lar_cache_host_join (or four

@@ -73,6 +73,7 @@ struct StreamArgs {
     int seq, need_seq;  // sequence number of this launch on its cache / of the launch that last wrote this layer's cache
     int* done_seq;      // device word: every launch up to this number has completed
     int q_slots, p_bufs;  // depth of the CTA's query ring / number of partial buffers
+    int stall_test;     // test hook: the producers issue no copy, so that the consumers' bounded waits run out
     int pool_row_base;  // first pool row of this layer in the tensor maps
     // elements between consecutive sequences of q / k_new / v_new / out (0: dense, heads of a sequence back to back and
     // sequences back to back); within a sequence the heads are always back to back
@@ -367,7 +368,9 @@ __global__ void __launch_bounds__(288, 1) decode_stream_kernel(const StreamArgs 
             fill_end = n_tiles < NS ? n_tiles : NS;
         }
         bool dep_waited = false;
-        const int n_local = n_tiles > pw ? (n_tiles - pw + kProducers - 1) / kProducers : 0;
+        // (test hook stall_test: the producers have nothing to request; the consumers' waits for their first tiles run
+        // into the limit and the launch ends with the wait-limit status bit)
+        const int n_local = (n_tiles > pw && !a.stall_test) ? (n_tiles - pw + kProducers - 1) / kProducers : 0;
 
         auto describe = [&](int jj, int& y, int& rows, int& tile) {
             const int t = t_begin + jj;

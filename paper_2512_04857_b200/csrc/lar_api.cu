@@ -554,6 +554,7 @@ lar_status_t launch_decode(lar_cache* c, int layer, const void* q, const void* k
         c->last_writer[layer] = a.seq;
         a.done_seq = reinterpret_cast<int*>(c->slab + c->L.off_status + 128);
         a.q_slots = c->d.q_slots;
+        a.stall_test = (c->cfg.flags & LAR_FLAG_TEST_STALL) ? 1 : 0;
         a.p_bufs = c->d.p_bufs;
         a.pool_row_base = layer * c->rows_per_layer;
         a.q_seq_stride = ss.q;

@@ -21,6 +21,7 @@ LAR_FLAG_SCORE_CACHE_NORM = 0x10
 LAR_FLAG_HOST_DEFER_OUT = 0x20
 LAR_FLAG_SCORE_ACCUM = 0x40
 LAR_FLAG_SLOT_REUSE = 0x80
+LAR_FLAG_TEST_STALL = 0x100
 
 
 class lar_config_t(C.Structure):

@@ -442,3 +442,37 @@ def test_softmax_scale_override_and_single_row_cache():
     ref = p[..., :1] * b["v"].double() + p[..., 1:] * v2.double()
     assert torch.allclose(b["out"].double(), ref, atol=1e-5)
     c.close()
+
+
+def test_a_wait_that_runs_out_ends_the_launch_with_a_status_bit_and_leaves_the_device_usable():
+    """Failure detection without a fault: with the test hook the producer warps request no tile, every consumer's
+    bounded wait for its first tile runs out (~1 s), the roles of each CTA give up and the launch returns by itself;
+    the host reads status bit 4.  A cache created afterwards works as usual."""
+    import time
+    cfg = _small(n_layers=1, flags=lar.LAR_FLAG_TEST_STALL)
+    c = lar.Cache(cfg)
+    b = _bufs(cfg)
+    c.append_kv(0, b["kc"], b["vc"], 4)
+    torch.cuda.synchronize()
+    t0 = time.time()
+    c.decode_step(0, b["q"], b["k"], b["v"], b["out"])
+    torch.cuda.synchronize()
+    dt = time.time() - t0
+    assert 0.5 < dt < 20.0, dt                       # the limit, not a hang and not an immediate return
+    bits = c.poll_device_status()
+    assert bits & 4, bits
+    c.close()
+    # the same device, a cache without the hook: a fused step agrees with the unfused append + attention of another cache
+    cfg2 = _small(n_layers=1)
+    c1, c2 = lar.Cache(cfg2), lar.Cache(cfg2)
+    o1, o2 = torch.zeros_like(b["out"]), torch.zeros_like(b["out"])
+    for cc in (c1, c2):
+        cc.append_kv(0, b["kc"], b["vc"], 4)
+    c1.decode_step(0, b["q"], b["k"], b["v"], o1)
+    c2.append_kv(0, b["k"], b["v"], 1)
+    c2.decode_attn(0, b["q"], o2)
+    torch.cuda.synchronize()
+    assert c1.poll_device_status() == 0 and c2.poll_device_status() == 0
+    assert torch.isfinite(o1.float()).all() and (o1.float() - o2.float()).abs().max().item() < 2e-2
+    c1.close()
+    c2.close()
