@@ -146,11 +146,9 @@ bool derive(const lar_config_t* c, Derived& d) {
     // line end: one CTA per unit, 8 warps; few units with a large mid region get one warp per 16 guide rows (16..32 warps)
     d.le_threads = 256;
     d.le_guide_global = 0;
-    // (a column sum per warp over every live row -- accumulated attention, or the cache-normalised form without
-    // compaction -- stays at 8 warps so that it fits into shared memory)
-    const bool all_cols = (c->flags & LAR_FLAG_SCORE_ACCUM) ||
-                          ((c->flags & LAR_FLAG_SLOT_REUSE) && (c->flags & LAR_FLAG_SCORE_CACHE_NORM));
-    if (!all_cols && d.units <= 2 * kDefaultDecodeCtas && d.M >= 128) {
+    // (with a column sum per warp over every live row -- accumulated attention, or the cache-normalised form without
+    // compaction -- the plan takes warps away again until the CTA fits into shared memory)
+    if (d.units <= 2 * kDefaultDecodeCtas && d.M >= 128) {
         const int blocks = (c->line_width * d.group + 15) / 16;
         d.le_threads = 32 * (blocks < 16 ? 16 : blocks > 32 ? 32 : blocks);
     }
@@ -268,6 +266,12 @@ lar_status_t plan_query_impl(const lar_config_t* cfg, lar_plan_t* out, Derived* 
                                         d.le_guide_global);
     };
     p.line_end_smem_bytes = d.compressing ? le_bytes() : 0;
+    const bool all_cols = (cfg->flags & LAR_FLAG_SCORE_ACCUM) ||
+                          ((cfg->flags & LAR_FLAG_SLOT_REUSE) && (cfg->flags & LAR_FLAG_SCORE_CACHE_NORM));
+    while (all_cols && p.line_end_smem_bytes > 227 * 1024 && d.le_threads > 256) {
+        d.le_threads -= 32;  // one row of column sums (every live row) less
+        p.line_end_smem_bytes = le_bytes();
+    }
     if (p.line_end_smem_bytes > 227 * 1024 && cfg->dtype == LAR_BF16 &&
         !(cfg->flags & (LAR_FLAG_SCORE_CACHE_NORM | LAR_FLAG_SCORE_ACCUM))) {
         // a mid region too large to stage next to the guide rows: 8 warps, guide rows read from global memory
