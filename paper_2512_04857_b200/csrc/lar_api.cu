@@ -145,6 +145,13 @@ bool derive(const lar_config_t* c, Derived& d) {
     // A unit of T tiles is cut into at most ceil(T / floor(U T / P)) + 1 segments (never more than T or P).
     // line end: one CTA per unit, 8 warps; few units with a large mid region get one warp per 16 guide rows (16..32 warps)
     d.le_threads = 256;
+    // A short line against a small mid region (at most two 16-row blocks of guide rows, 64 mid keys) is a chain of
+    // short block-wide phases: smaller CTAs, and so more of them per SM, hide its latencies better (measured per
+    // generation: 14.9 -> 11.5 ms on the Janus-Pro-7B shape with 4 warps, 17.2 -> 9.6 ms on the LlamaGen-XL shape with 2)
+    // (the written form of Eq. 9 only: the variants that stage the whole live cache have enough work for 8 warps)
+    if (c->dtype == LAR_BF16 && c->line_width * d.group <= 32 && d.M <= 64 &&
+        !(c->flags & (LAR_FLAG_SCORE_CACHE_NORM | LAR_FLAG_SCORE_ACCUM)))
+        d.le_threads = d.row_bytes <= 128 ? 64 : 128;
     d.le_guide_global = 0;
     // (with a column sum per warp over every live row -- accumulated attention, or the cache-normalised form without
     // compaction -- the plan takes warps away again until the CTA fits into shared memory)

@@ -150,7 +150,12 @@ def test_cache_normalised_scoring_plan():
         if w.dtype == "bf16":   # keys grow by extra_rows padded rows; the staged guide rows go away
             nq16 = (w.line_width * w.group + 15) // 16 * 16
             row = w.head_dim * 2 + 16
-            assert abs((var.line_end_smem_bytes - base.line_end_smem_bytes) - (extra_rows - nq16) * row) <= 16, name
+            # (a short line against a small mid region runs 2 or 4 warps in the written form, 8 in the variant: one row of
+            # M column sums per warp)
+            small = w.line_width * w.group <= 32 and w.mid_len <= 64
+            warps_base = (2 if w.head_dim * 2 <= 128 else 4) if small else None
+            colsums = (8 - warps_base) * w.mid_len * 4 if small else 0
+            assert abs((var.line_end_smem_bytes - base.line_end_smem_bytes) - (extra_rows - nq16) * row - colsums) <= 16, name
     big = W.WORKLOADS["gqa_1024"].scaled(score_norm="cache", cond_len=512)     # 1032 keys of 272 B > 227 KB
     with pytest.raises(lar.LarError) as e:
         lar.lar_plan_query(lar.config_from_workload(big))
